@@ -1,0 +1,197 @@
+"""ctypes front end of the fp64 CPU oracle (``zz_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY.  Used by ``tests/``, by the smoke check and by the timed
+CPU-baseline leg of ``bench.py``; the CUDA library and its Python binding never
+import this package, and this package imports nothing from them.  All arithmetic
+lives in the C file; this module only marshals numpy arrays (bf16 values travel as
+their 16-bit patterns in ``uint16`` arrays) and keeps per-sequence bookkeeping.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "zz_oracle.c")
+_LIB = os.path.join(_HERE, "libzz_oracle.so")
+_lib: Optional[ctypes.CDLL] = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP over independent (row, head) units)."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", _LIB, _SRC, "-lm"]
+    subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load() -> ctypes.CDLL:
+    global _lib
+    if _lib is not None:
+        return _lib
+    build()
+    lib = ctypes.CDLL(_LIB)
+    i64, i32, dbl, vp = ctypes.c_int64, ctypes.c_int, ctypes.c_double, ctypes.c_void_p
+    lib.zzo_visible.argtypes = [i32, i64, i64, i64, i64]
+    lib.zzo_visible.restype = i32
+    lib.zzo_visible_count.argtypes = [i32, i64, i64, i64]
+    lib.zzo_visible_count.restype = i64
+    lib.zzo_slot.argtypes = [i64, i64, i64]
+    lib.zzo_slot.restype = i64
+    lib.zzo_attn_rows.argtypes = [vp, vp, i64, vp, vp, i64, i32, i32, i32, vp, i64, i64, dbl, vp, vp]
+    lib.zzo_attn_rows.restype = i32
+    lib.zzo_ring_append.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, i32, i64, i64]
+    lib.zzo_ring_append.restype = i32
+    lib.zzo_full_append.argtypes = [vp, vp, i64, vp, vp, vp, i64, i32, i32]
+    lib.zzo_full_append.restype = i32
+    lib.zzo_attn_from_slots.argtypes = [vp, i64, vp, vp, vp, i64, i32, i32, i32, vp, i64, i64, dbl, vp]
+    lib.zzo_attn_from_slots.restype = i32
+    lib.zzo_num_threads.restype = i32
+    _lib = lib
+    return lib
+
+
+def _u16(a: np.ndarray) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    if a.dtype != np.uint16:
+        raise TypeError("bf16 tensors travel as uint16 bit patterns")
+    return a
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def num_threads() -> int:
+    return int(_load().zzo_num_threads())
+
+
+def visible(kind: int, j: int, t: int, S: int, W: int) -> bool:
+    return bool(_load().zzo_visible(int(kind), int(j), int(t), int(S), int(W)))
+
+
+def visible_count(kind: int, t: int, S: int, W: int) -> int:
+    return int(_load().zzo_visible_count(int(kind), int(t), int(S), int(W)))
+
+
+def slot(t: int, S: int, W: int) -> int:
+    return int(_load().zzo_slot(int(t), int(S), int(W)))
+
+
+def attn_rows(q: np.ndarray, t_rows: Sequence[int], k: np.ndarray, v: np.ndarray,
+              kv_kind: Sequence[int], S: int, W: int, scale: float,
+              return_psum: bool = False):
+    """Rows of attention from the full history.
+
+    q [n_rows, Hq, D] (row i is the query at absolute position t_rows[i]),
+    k, v [n_hist, Hkv, D], kv_kind [Hkv] (1 retrieval / 0 streaming).
+    Returns out [n_rows, Hq, D] float64 (and the per-row softmax weight sums)."""
+    q, k, v = _u16(q), _u16(k), _u16(v)
+    n_rows, Hq, D = q.shape
+    n_hist, Hkv, D2 = k.shape
+    assert D == D2 and v.shape == k.shape
+    t = np.ascontiguousarray(np.asarray(t_rows, dtype=np.int64))
+    assert t.shape == (n_rows,)
+    kinds = np.ascontiguousarray(np.asarray(kv_kind, dtype=np.uint8))
+    assert kinds.shape == (Hkv,)
+    out = np.empty((n_rows, Hq, D), dtype=np.float64)
+    psum = np.empty((n_rows, Hq), dtype=np.float64) if return_psum else None
+    rc = _load().zzo_attn_rows(_ptr(q), _ptr(t), n_rows, _ptr(k), _ptr(v), n_hist, Hq, Hkv, D,
+                               _ptr(kinds), int(S), int(W), float(scale), _ptr(out), _ptr(psum))
+    if rc != 0:
+        raise ValueError(f"zzo_attn_rows failed: {rc}")
+    return (out, psum) if return_psum else out
+
+
+def attn_from_slots(q: np.ndarray, t: int, store_k: np.ndarray, store_v: np.ndarray,
+                    pos: np.ndarray, kv_kind: Sequence[int], S: int, W: int,
+                    scale: float) -> np.ndarray:
+    """One row from a slot store: q [Hq, D], store_k/v [Hkv, n_slots, D], pos [n_slots]."""
+    q, store_k, store_v = _u16(q), _u16(store_k), _u16(store_v)
+    Hq, D = q.shape
+    Hkv, n_slots, _ = store_k.shape
+    pos = np.ascontiguousarray(pos, dtype=np.int32)
+    kinds = np.ascontiguousarray(np.asarray(kv_kind, dtype=np.uint8))
+    out = np.empty((Hq, D), dtype=np.float64)
+    rc = _load().zzo_attn_from_slots(_ptr(q), int(t), _ptr(store_k), _ptr(store_v), _ptr(pos),
+                                     n_slots, Hq, Hkv, D, _ptr(kinds), int(S), int(W),
+                                     float(scale), _ptr(out))
+    if rc != 0:
+        raise ValueError(f"zzo_attn_from_slots failed: {rc}")
+    return out
+
+
+class RingStore:
+    """Streaming KV store of one (layer, sequence): S+W slots, simulated token by token."""
+
+    def __init__(self, Hkv: int, D: int, S: int, W: int):
+        self.Hkv, self.D, self.S, self.W = Hkv, D, S, W
+        self.k = np.zeros((Hkv, S + W, D), dtype=np.uint16)
+        self.v = np.zeros((Hkv, S + W, D), dtype=np.uint16)
+        self.pos = np.full(S + W, -1, dtype=np.int32)
+        self._len = ctypes.c_int64(0)
+
+    @property
+    def len(self) -> int:
+        return int(self._len.value)
+
+    def append(self, k_new: np.ndarray, v_new: np.ndarray) -> None:
+        k_new, v_new = _u16(k_new), _u16(v_new)
+        C = k_new.shape[0]
+        assert k_new.shape == (C, self.Hkv, self.D) and v_new.shape == k_new.shape
+        rc = _load().zzo_ring_append(_ptr(self.k), _ptr(self.v), _ptr(self.pos),
+                                     ctypes.byref(self._len), _ptr(k_new), _ptr(v_new), C,
+                                     self.Hkv, self.D, self.S, self.W)
+        if rc != 0:
+            raise ValueError(f"zzo_ring_append failed: {rc}")
+
+
+class FullStore:
+    """Retrieval KV store of one (layer, sequence): slot j holds token j."""
+
+    def __init__(self, Hkv: int, D: int, cap: int):
+        self.Hkv, self.D, self.cap = Hkv, D, cap
+        self.k = np.zeros((Hkv, cap, D), dtype=np.uint16)
+        self.v = np.zeros((Hkv, cap, D), dtype=np.uint16)
+        self._len = ctypes.c_int64(0)
+
+    @property
+    def len(self) -> int:
+        return int(self._len.value)
+
+    @property
+    def pos(self) -> np.ndarray:
+        p = np.full(self.cap, -1, dtype=np.int32)
+        p[: self.len] = np.arange(self.len, dtype=np.int32)
+        return p
+
+    def append(self, k_new: np.ndarray, v_new: np.ndarray) -> None:
+        k_new, v_new = _u16(k_new), _u16(v_new)
+        C = k_new.shape[0]
+        rc = _load().zzo_full_append(_ptr(self.k), _ptr(self.v), self.cap,
+                                     ctypes.byref(self._len), _ptr(k_new), _ptr(v_new), C,
+                                     self.Hkv, self.D)
+        if rc != 0:
+            raise ValueError(f"zzo_full_append failed: {rc}")
+
+
+class History:
+    """Whole K/V history of one (layer, sequence), nothing waived: a growing array."""
+
+    def __init__(self, Hkv: int, D: int):
+        self.k = np.zeros((0, Hkv, D), dtype=np.uint16)
+        self.v = np.zeros((0, Hkv, D), dtype=np.uint16)
+
+    @property
+    def len(self) -> int:
+        return int(self.k.shape[0])
+
+    def append(self, k_new: np.ndarray, v_new: np.ndarray) -> None:
+        self.k = np.concatenate([self.k, _u16(k_new)], axis=0)
+        self.v = np.concatenate([self.v, _u16(v_new)], axis=0)

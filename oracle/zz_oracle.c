@@ -1,0 +1,245 @@
+/*
+ * CPU oracle for the ZigzagAttention inference hot path.  TEST INFRASTRUCTURE ONLY:
+ * it is used by the tests, by the smoke check and by the timed CPU-baseline leg of
+ * the benchmark; the product (the CUDA library) never calls, links or imports it,
+ * and it shares no code, header, table or helper with the CUDA path.
+ *
+ * Everything here is the plain definition written out, in fp64 on the bf16 input
+ * values widened exactly: no tiling, no online softmax, no reordering.
+ *
+ * What it computes (citations are to the paper):
+ *   - "full attention" of a retrieval head and "streaming attention" of a
+ *     streaming head (Section 2.1, the two terms of Eq. 1; Eq. 1 with alpha = 1
+ *     is the former and alpha = 0 the latter).  Streaming attention attends to the
+ *     sink tokens plus a recent window, the remaining KV being waived
+ *     (Introduction, the paragraph on DuoAttention; sink/window sizes are the two
+ *     hyper-parameters fixed in Section 3.3).
+ *   - the prefill and decoding phases over a KV cache (Introduction, second
+ *     paragraph): a prefill call evaluates rows t = P .. P+C-1, a decode step the
+ *     single row t = N-1 after the new token has been appended.
+ *   - the per-layer exclusive assignment (Section 2.2, first paragraph) is the
+ *     special case in which every KV head of the layer has the same kind; the
+ *     mixed-head (DuoAttention-style) layer is the general case, kind per KV head.
+ *
+ * Readings where the paper is silent (also listed in the design notes):
+ *   - visible set of a streaming head for the query at absolute position t:
+ *       V(t) = { j : 0 <= j <= t  and  ( j < S  or  t - j < W ) }
+ *     i.e. the window of W keys includes the current token;
+ *   - the streaming KV store is a ring of S+W slots: slot(t) = t for t < S,
+ *     otherwise S + ((t - S) mod W); pos[slot] holds the token index or -1;
+ *   - query head h uses KV head floor(h / G), G = Hq / Hkv;
+ *   - natural-base softmax with an explicit scale factor.
+ *
+ * Pins (see tests): brute force with an explicit score/mask matrix written
+ * differently (numpy, long double, no max subtraction); rows of the softmax sum to
+ * one; q = 0 gives the arithmetic mean of the visible values; a dominant key
+ * selects its value; S+W >= N equals full attention bit for bit; S=0, W=1 gives
+ * v_t; |V(t)| = min(t+1, S+W); decode step t == prefill row t; chunked == single
+ * shot; ring route == full-history route; occupied ring positions; invariance
+ * under slot permutation; GQA replication; mixed layer == per-head kinds.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ZZO_OK 0
+#define ZZO_BAD_ARG (-1)
+
+static double bf16_to_f64(uint16_t b) {
+    uint32_t u = ((uint32_t)b) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* V(t) membership.  kind: 1 = retrieval (full attention), 0 = streaming. */
+int zzo_visible(int kind, int64_t j, int64_t t, int64_t S, int64_t W) {
+    if (j < 0 || j > t) return 0;
+    if (kind) return 1;
+    return (j < S) || (t - j < W);
+}
+
+/* |V(t)| counted one key at a time. */
+int64_t zzo_visible_count(int kind, int64_t t, int64_t S, int64_t W) {
+    int64_t n = 0;
+    for (int64_t j = 0; j <= t; ++j) n += zzo_visible(kind, j, t, S, W);
+    return n;
+}
+
+/* Ring slot of token t (streaming KV store). */
+int64_t zzo_slot(int64_t t, int64_t S, int64_t W) {
+    if (t < S) return t;
+    return S + ((t - S) % W);
+}
+
+/*
+ * Attention rows from the full K/V history.
+ *   q        [n_rows][Hq][D]   bf16 bits, row i is the query at absolute position t_rows[i]
+ *   k, v     [n_hist][Hkv][D]  bf16 bits, token j at index j (the whole history, nothing waived)
+ *   kv_kind  [Hkv]             1 = retrieval KV head, 0 = streaming KV head
+ *   out      [n_rows][Hq][D]   fp64
+ *   p_sum    NULL or [n_rows][Hq]: the sum of the softmax weights of the row (should be 1)
+ * For each (row, head): s_j = scale * <q, k_j> over j in V(t); m = max s_j;
+ * p_j = exp(s_j - m) / sum_i exp(s_i - m); o = sum_j p_j v_j.
+ */
+int zzo_attn_rows(const uint16_t* q, const int64_t* t_rows, int64_t n_rows,
+                  const uint16_t* k, const uint16_t* v, int64_t n_hist,
+                  int Hq, int Hkv, int D, const uint8_t* kv_kind,
+                  int64_t S, int64_t W, double scale, double* out, double* p_sum) {
+    if (!q || !t_rows || !k || !v || !kv_kind || !out) return ZZO_BAD_ARG;
+    if (Hq <= 0 || Hkv <= 0 || D <= 0 || Hq % Hkv != 0 || n_rows < 0) return ZZO_BAD_ARG;
+    if (S < 0 || W < 1) return ZZO_BAD_ARG;
+    for (int64_t i = 0; i < n_rows; ++i)
+        if (t_rows[i] < 0 || t_rows[i] >= n_hist) return ZZO_BAD_ARG;
+    const int G = Hq / Hkv;
+    const int64_t units = n_rows * (int64_t)Hq;
+#pragma omp parallel
+    {
+        double* s = (double*)malloc(sizeof(double) * (size_t)(n_hist > 0 ? n_hist : 1));
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t u = 0; u < units; ++u) {
+            const int64_t i = u / Hq;
+            const int h = (int)(u % Hq);
+            const int g = h / G;
+            const int kind = kv_kind[g] ? 1 : 0;
+            const int64_t t = t_rows[i];
+            const uint16_t* qrow = q + ((size_t)i * Hq + h) * D;
+            /* scores and their maximum over the visible set */
+            double m = -INFINITY;
+            for (int64_t j = 0; j <= t; ++j) {
+                if (!zzo_visible(kind, j, t, S, W)) continue;
+                const uint16_t* krow = k + ((size_t)j * Hkv + g) * D;
+                double dot = 0.0;
+                for (int d = 0; d < D; ++d) dot += bf16_to_f64(qrow[d]) * bf16_to_f64(krow[d]);
+                s[j] = scale * dot;
+                if (s[j] > m) m = s[j];
+            }
+            /* normaliser */
+            double denom = 0.0;
+            for (int64_t j = 0; j <= t; ++j) {
+                if (!zzo_visible(kind, j, t, S, W)) continue;
+                denom += exp(s[j] - m);
+            }
+            /* weighted sum of the values */
+            double* orow = out + ((size_t)i * Hq + h) * D;
+            for (int d = 0; d < D; ++d) orow[d] = 0.0;
+            double psum = 0.0;
+            for (int64_t j = 0; j <= t; ++j) {
+                if (!zzo_visible(kind, j, t, S, W)) continue;
+                const double p = exp(s[j] - m) / denom;
+                psum += p;
+                const uint16_t* vrow = v + ((size_t)j * Hkv + g) * D;
+                for (int d = 0; d < D; ++d) orow[d] += p * bf16_to_f64(vrow[d]);
+            }
+            if (p_sum) p_sum[(size_t)i * Hq + h] = psum;
+        }
+        free(s);
+    }
+    return ZZO_OK;
+}
+
+/*
+ * Streaming KV store: append C tokens one at a time to a ring of S+W slots.
+ *   ring_k, ring_v [Hkv][S+W][D]  bf16 bits (canonical export order)
+ *   pos            [S+W]          token index held by the slot, -1 = empty
+ *   len            in/out         tokens appended so far
+ *   k_new, v_new   [C][Hkv][D]
+ * Token t goes to slot(t); whatever was there (token t - W) is thereby evicted.
+ */
+int zzo_ring_append(uint16_t* ring_k, uint16_t* ring_v, int32_t* pos, int64_t* len,
+                    const uint16_t* k_new, const uint16_t* v_new, int64_t C,
+                    int Hkv, int D, int64_t S, int64_t W) {
+    if (!ring_k || !ring_v || !pos || !len || (C > 0 && (!k_new || !v_new))) return ZZO_BAD_ARG;
+    if (Hkv <= 0 || D <= 0 || S < 0 || W < 1 || C < 0) return ZZO_BAD_ARG;
+    const int64_t R = S + W;
+    for (int64_t i = 0; i < C; ++i) {
+        const int64_t t = *len;
+        const int64_t sl = zzo_slot(t, S, W);
+        for (int g = 0; g < Hkv; ++g) {
+            memcpy(ring_k + ((size_t)g * R + sl) * D, k_new + ((size_t)i * Hkv + g) * D,
+                   sizeof(uint16_t) * (size_t)D);
+            memcpy(ring_v + ((size_t)g * R + sl) * D, v_new + ((size_t)i * Hkv + g) * D,
+                   sizeof(uint16_t) * (size_t)D);
+        }
+        pos[sl] = (int32_t)t;
+        *len = t + 1;
+    }
+    return ZZO_OK;
+}
+
+/*
+ * Retrieval KV store: slot j holds token j.
+ *   cache_k, cache_v [Hkv][cap][D]; len in/out; returns ZZO_BAD_ARG on overflow
+ *   (and leaves everything unchanged).
+ */
+int zzo_full_append(uint16_t* cache_k, uint16_t* cache_v, int64_t cap, int64_t* len,
+                    const uint16_t* k_new, const uint16_t* v_new, int64_t C, int Hkv, int D) {
+    if (!cache_k || !cache_v || !len || (C > 0 && (!k_new || !v_new))) return ZZO_BAD_ARG;
+    if (*len + C > cap || C < 0) return ZZO_BAD_ARG;
+    for (int64_t i = 0; i < C; ++i) {
+        const int64_t t = *len;
+        for (int g = 0; g < Hkv; ++g) {
+            memcpy(cache_k + ((size_t)g * cap + t) * D, k_new + ((size_t)i * Hkv + g) * D,
+                   sizeof(uint16_t) * (size_t)D);
+            memcpy(cache_v + ((size_t)g * cap + t) * D, v_new + ((size_t)i * Hkv + g) * D,
+                   sizeof(uint16_t) * (size_t)D);
+        }
+        *len = t + 1;
+    }
+    return ZZO_OK;
+}
+
+/*
+ * One attention row computed from a slot store (ring or retrieval cache) instead
+ * of the history: every slot with pos >= 0 holds token pos[slot]; the key takes
+ * part iff pos[slot] is in V(t).  Slots are visited in physical order.
+ *   q [Hq][D]; store_k, store_v [Hkv][n_slots][D]; pos [n_slots]; out [Hq][D] fp64
+ */
+int zzo_attn_from_slots(const uint16_t* q, int64_t t, const uint16_t* store_k,
+                        const uint16_t* store_v, const int32_t* pos, int64_t n_slots,
+                        int Hq, int Hkv, int D, const uint8_t* kv_kind,
+                        int64_t S, int64_t W, double scale, double* out) {
+    if (!q || !store_k || !store_v || !pos || !kv_kind || !out) return ZZO_BAD_ARG;
+    if (Hq <= 0 || Hkv <= 0 || D <= 0 || Hq % Hkv != 0) return ZZO_BAD_ARG;
+    const int G = Hq / Hkv;
+    double* s = (double*)malloc(sizeof(double) * (size_t)(n_slots > 0 ? n_slots : 1));
+    for (int h = 0; h < Hq; ++h) {
+        const int g = h / G;
+        const int kind = kv_kind[g] ? 1 : 0;
+        const uint16_t* qrow = q + (size_t)h * D;
+        double m = -INFINITY;
+        for (int64_t sl = 0; sl < n_slots; ++sl) {
+            if (pos[sl] < 0 || !zzo_visible(kind, pos[sl], t, S, W)) continue;
+            const uint16_t* krow = store_k + ((size_t)g * n_slots + sl) * D;
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d) dot += bf16_to_f64(qrow[d]) * bf16_to_f64(krow[d]);
+            s[sl] = scale * dot;
+            if (s[sl] > m) m = s[sl];
+        }
+        double denom = 0.0;
+        for (int64_t sl = 0; sl < n_slots; ++sl) {
+            if (pos[sl] < 0 || !zzo_visible(kind, pos[sl], t, S, W)) continue;
+            denom += exp(s[sl] - m);
+        }
+        double* orow = out + (size_t)h * D;
+        for (int d = 0; d < D; ++d) orow[d] = 0.0;
+        for (int64_t sl = 0; sl < n_slots; ++sl) {
+            if (pos[sl] < 0 || !zzo_visible(kind, pos[sl], t, S, W)) continue;
+            const double p = exp(s[sl] - m) / denom;
+            const uint16_t* vrow = store_v + ((size_t)g * n_slots + sl) * D;
+            for (int d = 0; d < D; ++d) orow[d] += p * bf16_to_f64(vrow[d]);
+        }
+    }
+    free(s);
+    return ZZO_OK;
+}
+
+int zzo_num_threads(void) {
+#ifdef _OPENMP
+    extern int omp_get_max_threads(void);
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
