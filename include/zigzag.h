@@ -1,0 +1,176 @@
+/*
+ * zigzag.h -- C ABI of the ZigzagAttention inference hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library runs the per-layer attention pass of a model whose layers are each
+ * exclusively "retrieval" (full causal attention over the whole KV cache) or
+ * exclusively "streaming" (attention to sink tokens plus a recent window, the rest of
+ * the KV waived), so that each layer needs one attention call (paper: Introduction,
+ * last-but-one paragraph; Section 2.2, first paragraph).  It also carries the
+ * DuoAttention-style layer that mixes both kinds of head in one layer and therefore
+ * runs two passes plus head gather/scatter (paper: Introduction, the paragraph on the
+ * cost of DuoAttention; Section 2.1, last paragraph) as the in-library comparison.
+ *
+ * Conventions
+ *   - Every function returns an int status: ZZ_OK (0) or a negative ZZ_ERR_* code.
+ *     Nothing throws or aborts across this boundary.  A call that fails argument or
+ *     capacity validation has launched nothing and leaves the cache unchanged.
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  The caller
+ *     allocates and owns all device memory (tensors, the cache arena, the workspace);
+ *     the library owns only the small host-side handle.  Unless stated otherwise the
+ *     library never allocates or frees device memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All
+ *     compute calls are asynchronous on that stream.  A handle is not thread-safe and
+ *     calls on one handle must be issued in stream order on one stream at a time.
+ *   - Tensors are bf16 (2-byte), row-major, innermost dimension head_dim = 128.
+ *     q/out of a call:   [tokens, n_q_heads, head_dim]
+ *     k/v of a call:     [tokens, n_kv_heads, head_dim]
+ *     `tokens` is the packed concatenation over the batch, sequence 0 first.
+ *   - Query head h reads KV head h / (n_q_heads / n_kv_heads).
+ *   - Token positions are absolute and 0-based; a sequence's length `len` is the number
+ *     of tokens appended so far.  Lengths live on the device (so that a captured
+ *     sequence of calls can be replayed) and are mirrored on the host for validation.
+ *
+ * Visibility rule (S = sink, W = recent):
+ *   retrieval head:  the query at position t sees every key j <= t;
+ *   streaming head:  it sees key j <= t iff  j < S  or  t - j < W  (the window counts
+ *                    the current token).
+ * Streaming KV store: a ring of S+W slots per (layer, sequence, KV head);
+ *   slot(t) = t for t < S, else S + ((t - S) mod W); pos[slot] is the token held or -1.
+ * Retrieval KV store: slot j holds token j, up to capacity[seq] tokens.
+ */
+#ifndef ZIGZAG_H_
+#define ZIGZAG_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ZZ_OK 0
+#define ZZ_ERR_INVALID_ARG (-1) /* NULL pointer, index out of range, inconsistent sizes        */
+#define ZZ_ERR_UNSUPPORTED (-2) /* head_dim != 128, group size > 16, batch > ZZ_MAX_BATCH, ...  */
+#define ZZ_ERR_CAPACITY (-3)    /* len + n_new would exceed capacity[seq] of a retrieval store  */
+#define ZZ_ERR_WORKSPACE (-4)   /* arena or workspace smaller than zz_cache_query reported      */
+#define ZZ_ERR_CUDA (-5)        /* a CUDA runtime/driver call failed                            */
+#define ZZ_ERR_TIMEOUT (-6)     /* a bounded device-side wait expired (see zz_get_last_status)  */
+
+#define ZZ_MAX_BATCH 64
+#define ZZ_KIND_STREAMING 0
+#define ZZ_KIND_RETRIEVAL 1
+
+typedef struct zz_cache zz_cache_t;
+
+/* Plain-data description of the attention stack.  All pointers are HOST pointers and
+ * are only read during zz_cache_query / zz_cache_create. */
+typedef struct zz_config {
+    int32_t n_layers;
+    int32_t batch;                      /* sequences, 1 .. ZZ_MAX_BATCH                         */
+    int32_t n_q_heads;
+    int32_t n_kv_heads;                 /* divides n_q_heads; group size <= 16                  */
+    int32_t head_dim;                   /* must be 128                                          */
+    int32_t sink;                       /* S >= 0                                               */
+    int32_t recent;                     /* W >= 1                                               */
+    int32_t max_new_tokens;             /* largest sum of n_new over the batch in one prefill
+                                           call (sizes the mixed-layer gather buffers); >= batch */
+    float softmax_scale;                /* e.g. 1/sqrt(128)                                     */
+    const uint8_t* layer_is_retrieval;  /* [n_layers]  the exclusive per-layer mask             */
+    const uint8_t* kvhead_is_retrieval; /* NULL, or [n_layers * n_kv_heads]: per-KV-head kinds
+                                           (overrides the layer mask; a layer holding both
+                                           kinds runs the two-pass mixed-head path)             */
+    const int32_t* capacity;            /* [batch] max tokens per sequence in retrieval stores  */
+} zz_config_t;
+
+/* Library version (major*10000 + minor*100 + patch). */
+int zz_version(void);
+/* Static, NUL-terminated description of a status code. */
+const char* zz_status_str(int status);
+
+/* Bytes the caller must provide for the KV arena and the workspace (both device memory,
+ * 256-byte aligned).  Cache layout: paper, Introduction (KV cache of the prefill and decoding phases); streaming
+ * stores keep only sink + recent entries (Introduction; Section 3.3 for the sizes). */
+int zz_cache_query(const zz_config_t* cfg, size_t* arena_bytes, size_t* workspace_bytes);
+
+/* Builds the handle on caller-provided device memory, zero-fills the arena, sets all
+ * lengths to 0 and all ring positions to -1.  Synchronous (returns after the device
+ * finished initialising).  *out is written only on success. */
+int zz_cache_create(const zz_config_t* cfg, void* d_arena, size_t arena_bytes, void* d_workspace,
+                    size_t workspace_bytes, zz_cache_t** out);
+/* Frees the host handle (device memory stays the caller's). */
+int zz_cache_destroy(zz_cache_t* cache);
+/* Forgets the tokens of sequence `seq` (-1: all sequences) in every layer. */
+int zz_cache_reset(zz_cache_t* cache, int seq, void* stream);
+/* Host-mirrored length of (layer, seq). */
+int zz_cache_len(const zz_cache_t* cache, int layer, int seq, int32_t* len);
+
+/* Tuning knob for experiments; the paper has no counterpart.  Keys: "decode_min_chunk"
+ * (fewest tokens per split of the decode kernel; a multiple of 16, default 256). */
+int zz_tune(zz_cache_t* cache, const char* key, int value);
+
+/* KV append with sink + recent eviction (paper: Introduction -- the KV cache grows with
+ * the tokens seen; streaming heads waive all but sink and recent entries).
+ * Appends h_n_new[b] tokens of sequence b to `layer`: retrieval stores take token t in
+ * slot t; streaming stores take it in slot(t), overwriting token t - W.  d_k/d_v are
+ * packed [sum n_new, n_kv_heads, 128].  Fails with ZZ_ERR_CAPACITY (nothing written)
+ * if any retrieval store would overflow. */
+int zz_kv_append(zz_cache_t* cache, int layer, const void* d_k, const void* d_v,
+                 const int32_t* h_n_new, void* stream);
+
+/* Prefill attention of one layer (paper: Introduction, prefilling phase; Section 2.1, the
+ * two kinds of attention).  For sequence b the h_n_new[b] new queries sit at positions
+ * len .. len+n_new-1 and attend over (the store as it stands) U (the new chunk d_k/d_v)
+ * under the visibility rule of their head's kind.  The store is NOT modified: append the
+ * same chunk afterwards with zz_kv_append (attend-then-append, so a chunk longer than the
+ * window never evicts keys its own early rows need).  d_q/d_out are packed
+ * [sum n_new, n_q_heads, 128]; d_k/d_v packed [sum n_new, n_kv_heads, 128]; all four must
+ * be 16-byte aligned. */
+int zz_prefill_attn(zz_cache_t* cache, int layer, const void* d_q, const void* d_k,
+                    const void* d_v, void* d_out, const int32_t* h_n_new, void* stream);
+
+/* Decode attention of one layer (paper: Introduction, decoding phase): one query per
+ * sequence, at position len-1, over the store, which must already hold that token.
+ * d_q/d_out: [batch, n_q_heads, 128]. */
+int zz_decode_attn(zz_cache_t* cache, int layer, const void* d_q, void* d_out, void* stream);
+
+/* zz_kv_append of one token per sequence followed by zz_decode_attn. */
+int zz_decode_step(zz_cache_t* cache, int layer, const void* d_q, const void* d_k,
+                   const void* d_v, void* d_out, void* stream);
+
+/* The same two calls fed from HOST memory: copies q/k/v into caller-provided device
+ * staging (d_stage, at least zz_stage_bytes(cache, n_tokens) bytes), runs the call and
+ * copies the result back to h_out.  Pinned host memory makes the copies asynchronous.
+ * Prefill also appends the chunk after attending. */
+size_t zz_stage_bytes(const zz_cache_t* cache, int64_t n_tokens);
+int zz_decode_step_host(zz_cache_t* cache, int layer, const void* h_q, const void* h_k,
+                        const void* h_v, void* h_out, void* d_stage, size_t stage_bytes,
+                        void* stream);
+int zz_prefill_host(zz_cache_t* cache, int layer, const void* h_q, const void* h_k,
+                    const void* h_v, void* h_out, const int32_t* h_n_new, void* d_stage,
+                    size_t stage_bytes, void* stream);
+
+/* Snapshot of one store, for tests and checkpointing.  `kind` selects the KV-head group
+ * of the layer (ZZ_KIND_RETRIEVAL / ZZ_KIND_STREAMING; an exclusive layer has only one).
+ * h_k/h_v receive [n_heads_of_kind, n_slots, 128] bf16 in ascending KV-head order, where
+ * n_slots = capacity[seq] (retrieval) or S+W (streaming); h_pos [n_slots] receives the
+ * token held by each slot or -1; *h_len the length.  zz_cache_export_shape reports
+ * n_heads_of_kind and n_slots.  Both synchronise the stream. */
+int zz_cache_export_shape(const zz_cache_t* cache, int layer, int seq, int kind,
+                          int32_t* n_heads, int32_t* n_slots);
+int zz_cache_export(zz_cache_t* cache, int layer, int seq, int kind, void* h_k, void* h_v,
+                    int32_t* h_pos, int32_t* h_len, void* stream);
+/* Inverse of zz_cache_export for one group; sets the length of (layer, seq) to `len`. */
+int zz_cache_import(zz_cache_t* cache, int layer, int seq, int kind, const void* h_k,
+                    const void* h_v, const int32_t* h_pos, int32_t len, void* stream);
+
+/* Reads (and clears) the device status word: ZZ_OK, or ZZ_ERR_TIMEOUT if a bounded wait
+ * inside a kernel expired since the last read.  Synchronises the stream. */
+int zz_get_last_status(zz_cache_t* cache, void* stream);
+
+/* Number of kernels this library has launched since it was loaded (all handles). */
+int64_t zz_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZIGZAG_H_ */

@@ -1,0 +1,667 @@
+// C ABI of the library: handle, layout, validation and per-layer dispatch.
+// Every step of the hot path runs in the kernels of the sibling .cu files; this file only
+// checks arguments, plans launches and tracks lengths.
+#include <cuda.h>
+
+#include <atomic>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "zz_common.cuh"
+
+namespace zz {
+static std::atomic<long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+}  // namespace zz
+
+using zz::kD;
+using zz::SeqDesc;
+
+namespace {
+
+constexpr int kMaxSplits = 128;
+constexpr size_t kAlign = 256;
+
+size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+
+struct Layout {
+    // workspace sections (byte offsets)
+    size_t off_status, off_len, off_pos, off_desc, off_heads, off_counters, off_part_ml, off_part_o,
+        off_qc, off_oc, work_bytes;
+    size_t arena_bytes;
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// [rows][heads][128] bf16 seen as a 3-D tensor; a box is 128 rows x 1 head x 64 columns (128-byte swizzle)
+bool encode_rows3d(CUtensorMap* m, const void* base, long long rows, int heads) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)heads, (cuuint64_t)rows};
+    cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)heads * kD * 2};
+    cuuint32_t box[3] = {64, 1, 128};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// the arena as [rows][128] bf16; a box is 128 rows x 64 columns
+bool encode_rows2d(CUtensorMap* m, const void* base, long long rows) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
+    cuuint32_t box[2] = {64, 128};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+struct zz_cache {
+    int L, B, Hq, Hkv, G, S, W, ring, max_new;
+    float scale;
+    std::vector<uint8_t> kind;        // [L*Hkv]
+    std::vector<int> nR;              // [L] retrieval KV heads of the layer
+    std::vector<int> heads;           // [L*Hkv] group-ordered KV heads (retrieval first), ascending in each group
+    std::vector<int> cap;             // [B]
+    std::vector<int> len;             // [L*B] host mirror
+    std::vector<SeqDesc> desc;        // [L*B]
+    Layout lay;
+    unsigned char* arena;
+    unsigned char* work;
+    int num_sms;
+    int decode_min_chunk;
+    bool has_mixed;
+    alignas(64) CUtensorMap tmap_arena;
+    bool have_tmap_arena;
+
+    int* d_status() const { return reinterpret_cast<int*>(work + lay.off_status); }
+    unsigned int* d_append_counter() const { return reinterpret_cast<unsigned int*>(work + lay.off_status + 64); }
+    int* d_len(int l) const { return reinterpret_cast<int*>(work + lay.off_len) + (size_t)l * B; }
+    int* d_pos(int l) const { return reinterpret_cast<int*>(work + lay.off_pos) + (size_t)l * B * ring; }
+    SeqDesc* d_desc(int l) const { return reinterpret_cast<SeqDesc*>(work + lay.off_desc) + (size_t)l * B; }
+    int* d_heads(int l) const { return reinterpret_cast<int*>(work + lay.off_heads) + (size_t)l * Hkv; }
+    unsigned int* d_counters() const { return reinterpret_cast<unsigned int*>(work + lay.off_counters); }
+    float* d_part_ml() const { return reinterpret_cast<float*>(work + lay.off_part_ml); }
+    float* d_part_o() const { return reinterpret_cast<float*>(work + lay.off_part_o); }
+    __nv_bfloat16* d_qc() const { return reinterpret_cast<__nv_bfloat16*>(work + lay.off_qc); }
+    __nv_bfloat16* d_oc() const { return reinterpret_cast<__nv_bfloat16*>(work + lay.off_oc); }
+    __nv_bfloat16* d_arena() const { return reinterpret_cast<__nv_bfloat16*>(arena); }
+    bool mixed(int l) const { return nR[l] > 0 && nR[l] < Hkv; }
+};
+
+namespace {
+
+int validate(const zz_config_t* c) {
+    if (!c || !c->layer_is_retrieval || !c->capacity) return ZZ_ERR_INVALID_ARG;
+    if (c->n_layers < 1 || c->batch < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1) return ZZ_ERR_INVALID_ARG;
+    if (c->sink < 0 || c->recent < 1) return ZZ_ERR_INVALID_ARG;
+    if (c->max_new_tokens < c->batch) return ZZ_ERR_INVALID_ARG;
+    if (!(c->softmax_scale > 0.f)) return ZZ_ERR_INVALID_ARG;
+    if (c->head_dim != kD) return ZZ_ERR_UNSUPPORTED;
+    if (c->batch > ZZ_MAX_BATCH) return ZZ_ERR_UNSUPPORTED;
+    if (c->n_q_heads % c->n_kv_heads != 0) return ZZ_ERR_UNSUPPORTED;
+    if (c->n_q_heads / c->n_kv_heads > 16) return ZZ_ERR_UNSUPPORTED;
+    for (int b = 0; b < c->batch; ++b)
+        if (c->capacity[b] < 1) return ZZ_ERR_INVALID_ARG;
+    return ZZ_OK;
+}
+
+uint8_t kind_of(const zz_config_t* c, int l, int h) {
+    if (c->kvhead_is_retrieval) return c->kvhead_is_retrieval[(size_t)l * c->n_kv_heads + h] ? 1 : 0;
+    return c->layer_is_retrieval[l] ? 1 : 0;
+}
+
+// Arena: for each layer, for each sequence: retrieval group K [nR][cap][128], V likewise, then
+// streaming group K [nS][S+W][128], V likewise.  Fills `desc` if given.
+void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* desc) {
+    const int L = c->n_layers, B = c->batch, Hkv = c->n_kv_heads, Hq = c->n_q_heads;
+    const int ring = c->sink + c->recent;
+    const int G = Hq / Hkv;
+    long long off = 0;  // elements
+    bool has_mixed = false;
+    if (desc) desc->assign((size_t)L * B, SeqDesc());
+    for (int l = 0; l < L; ++l) {
+        int nR = 0;
+        for (int h = 0; h < Hkv; ++h) nR += kind_of(c, l, h);
+        const int nS = Hkv - nR;
+        if (nR > 0 && nS > 0) has_mixed = true;
+        for (int b = 0; b < B; ++b) {
+            SeqDesc d;
+            d.cap = c->capacity[b];
+            d.pad = 0;
+            d.k_off[ZZ_KIND_RETRIEVAL] = off;
+            off += (long long)nR * d.cap * kD;
+            d.v_off[ZZ_KIND_RETRIEVAL] = off;
+            off += (long long)nR * d.cap * kD;
+            d.k_off[ZZ_KIND_STREAMING] = off;
+            off += (long long)nS * ring * kD;
+            d.v_off[ZZ_KIND_STREAMING] = off;
+            off += (long long)nS * ring * kD;
+            if (desc) (*desc)[(size_t)l * B + b] = d;
+        }
+    }
+    // one spare tile of rows so that a 128-row tile read starting at the last valid row of the
+    // last store stays inside the tensor map's extent (out-of-extent rows read as zero anyway)
+    lay->arena_bytes = align_up((size_t)off * 2 + 128 * kD * 2);
+    size_t w = 0;
+    lay->off_status = w; w += kAlign;
+    lay->off_len = w; w += align_up((size_t)L * B * sizeof(int));
+    lay->off_pos = w; w += align_up((size_t)L * B * ring * sizeof(int));
+    lay->off_desc = w; w += align_up((size_t)L * B * sizeof(SeqDesc));
+    lay->off_heads = w; w += align_up((size_t)L * Hkv * sizeof(int));
+    lay->off_counters = w; w += align_up((size_t)B * Hkv * sizeof(unsigned int));
+    lay->off_part_ml = w; w += align_up((size_t)B * Hkv * kMaxSplits * G * 2 * sizeof(float));
+    lay->off_part_o = w; w += align_up((size_t)B * Hkv * kMaxSplits * G * kD * sizeof(float));
+    lay->off_qc = w;
+    if (has_mixed) w += align_up((size_t)c->max_new_tokens * Hq * kD * 2);
+    lay->off_oc = w;
+    if (has_mixed) w += align_up((size_t)c->max_new_tokens * Hq * kD * 2);
+    lay->work_bytes = w;
+}
+
+bool bad_layer(const zz_cache* c, int layer) { return !c || layer < 0 || layer >= c->L; }
+
+// Tokens per split and per-sequence split counts so that all work items fit one wave.
+void plan_splits(const zz_cache* c, const int* n, int Hg, int* chunk_out, int* split_start) {
+    const int slots = 2 * c->num_sms;
+    long long total = 0;
+    for (int b = 0; b < c->B; ++b) total += n[b];
+    long long chunk = (total * Hg + slots - 1) / slots;
+    chunk = (chunk + 63) / 64 * 64;
+    if (chunk < c->decode_min_chunk) chunk = c->decode_min_chunk;
+    for (;;) {
+        long long items = 0;
+        int worst = 0;
+        for (int b = 0; b < c->B; ++b) {
+            const int s = (int)((n[b] + chunk - 1) / chunk);
+            items += (long long)(s > 0 ? s : 1) * Hg;
+            if (s > worst) worst = s;
+        }
+        if ((items <= slots || chunk >= total) && worst <= kMaxSplits) break;
+        chunk += 64;
+    }
+    split_start[0] = 0;
+    for (int b = 0; b < c->B; ++b) {
+        int s = (int)((n[b] + chunk - 1) / chunk);
+        if (s < 1) s = 1;
+        split_start[b + 1] = split_start[b] + s;
+    }
+    *chunk_out = (int)chunk;
+}
+
+int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q, __nv_bfloat16* out,
+                        int q_head0, cudaStream_t st) {
+    const int Hg = (kind == ZZ_KIND_RETRIEVAL) ? c->nR[layer] : c->Hkv - c->nR[layer];
+    if (Hg == 0) return ZZ_OK;
+    zz::DecodeParams p;
+    memset(&p, 0, sizeof p);
+    p.arena = c->d_arena();
+    p.desc = c->d_desc(layer);
+    p.len = c->d_len(layer);
+    p.q = q;
+    p.out = out;
+    p.q_tok_stride = (long long)c->Hq * kD;
+    p.q_head0 = q_head0;
+    p.part_o = c->d_part_o();
+    p.part_ml = c->d_part_ml();
+    p.counters = c->d_counters();
+    p.status = c->d_status();
+    p.kind = kind;
+    p.ring = c->ring;
+    p.Hg = Hg;
+    p.G = c->G;
+    p.B = c->B;
+    p.max_splits = kMaxSplits;
+    p.scale_log2 = c->scale * 1.4426950408889634f;
+    int n[ZZ_MAX_BATCH];
+    for (int b = 0; b < c->B; ++b) {
+        const int len = c->len[(size_t)layer * c->B + b];
+        n[b] = (kind == ZZ_KIND_RETRIEVAL) ? len : (len < c->ring ? len : c->ring);
+    }
+    plan_splits(c, n, Hg, &p.chunk, p.split_start);
+    const int items = p.split_start[c->B] * Hg;
+    return zz::launch_decode(p, items, st) == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
+}
+
+int regroup(zz_cache* c, int layer, const __nv_bfloat16* src, __nv_bfloat16* dst, long long tokens,
+            int to_compact, cudaStream_t st) {
+    zz::GatherParams g;
+    g.src = src;
+    g.dst = dst;
+    g.head_list = c->d_heads(layer);
+    g.Hkv = c->Hkv;
+    g.G = c->G;
+    g.tokens = tokens;
+    g.to_compact = to_compact;
+    return zz::launch_regroup(g, st) == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
+}
+
+int launch_prefill_group(zz_cache* c, int layer, int kind, const CUtensorMap* tq, const CUtensorMap* tk,
+                         const CUtensorMap* tv, __nv_bfloat16* out, int q_head0, const int32_t* n_new,
+                         cudaStream_t st) {
+    const int nR = c->nR[layer];
+    const int Hg = (kind == ZZ_KIND_RETRIEVAL) ? nR : c->Hkv - nR;
+    if (Hg == 0) return ZZ_OK;
+    zz::PrefillParams p;
+    memset(&p, 0, sizeof p);
+    p.desc = c->d_desc(layer);
+    p.len = c->d_len(layer);
+    p.pos = c->d_pos(layer);
+    p.out = out;
+    p.tok_stride = (long long)c->Hq * kD;
+    p.head_list = c->d_heads(layer);
+    p.status = c->d_status();
+    p.kind = kind;
+    p.kv_head0 = (kind == ZZ_KIND_RETRIEVAL) ? 0 : nR;
+    p.q_head0 = q_head0;
+    p.n_kv_total = c->Hkv;
+    p.ring = c->ring;
+    p.S = c->S;
+    p.W = c->W;
+    p.Hg = Hg;
+    p.G = c->G;
+    p.B = c->B;
+    p.scale_log2 = c->scale * 1.4426950408889634f;
+    int off = 0, tiles = 0;
+    for (int b = 0; b < c->B; ++b) {
+        p.n_new[b] = n_new[b];
+        p.tok_off[b] = off;
+        p.tile_start[b] = tiles;
+        off += n_new[b];
+        tiles += (n_new[b] + 127) / 128;
+    }
+    p.tile_start[c->B] = tiles;
+    p.total_tiles = tiles;
+    const int pairs = (c->G + 1) / 2;
+    const long long items = (long long)tiles * Hg * pairs;
+    if (items == 0) return ZZ_OK;
+    if (items > 0x7fffffffLL) return ZZ_ERR_UNSUPPORTED;
+    return zz::launch_prefill(p, tq, tk, tv, &c->tmap_arena, (int)items, st) == cudaSuccess ? ZZ_OK
+                                                                                             : ZZ_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+int zz_version(void) { return 100; }
+
+const char* zz_status_str(int s) {
+    switch (s) {
+        case ZZ_OK: return "ok";
+        case ZZ_ERR_INVALID_ARG: return "invalid argument";
+        case ZZ_ERR_UNSUPPORTED: return "unsupported configuration";
+        case ZZ_ERR_CAPACITY: return "retrieval store capacity exceeded";
+        case ZZ_ERR_WORKSPACE: return "arena or workspace too small";
+        case ZZ_ERR_CUDA: return "CUDA error";
+        case ZZ_ERR_TIMEOUT: return "bounded device-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+int64_t zz_launch_count(void) { return zz::g_launches.load(std::memory_order_relaxed); }
+
+int zz_cache_query(const zz_config_t* cfg, size_t* arena_bytes, size_t* workspace_bytes) {
+    const int v = validate(cfg);
+    if (v != ZZ_OK) return v;
+    if (!arena_bytes || !workspace_bytes) return ZZ_ERR_INVALID_ARG;
+    Layout lay;
+    compute_layout(cfg, &lay, nullptr);
+    *arena_bytes = lay.arena_bytes;
+    *workspace_bytes = lay.work_bytes;
+    return ZZ_OK;
+}
+
+int zz_cache_create(const zz_config_t* cfg, void* d_arena, size_t arena_bytes, void* d_workspace,
+                    size_t workspace_bytes, zz_cache_t** out) {
+    const int v = validate(cfg);
+    if (v != ZZ_OK) return v;
+    if (!d_arena || !d_workspace || !out) return ZZ_ERR_INVALID_ARG;
+    if (((uintptr_t)d_arena % kAlign) || ((uintptr_t)d_workspace % kAlign)) return ZZ_ERR_INVALID_ARG;
+    zz_cache* c = new (std::nothrow) zz_cache();
+    if (!c) return ZZ_ERR_INVALID_ARG;
+    c->L = cfg->n_layers; c->B = cfg->batch; c->Hq = cfg->n_q_heads; c->Hkv = cfg->n_kv_heads;
+    c->G = c->Hq / c->Hkv; c->S = cfg->sink; c->W = cfg->recent; c->ring = c->S + c->W;
+    c->max_new = cfg->max_new_tokens; c->scale = cfg->softmax_scale;
+    c->decode_min_chunk = 256;
+    compute_layout(cfg, &c->lay, &c->desc);
+    if (arena_bytes < c->lay.arena_bytes || workspace_bytes < c->lay.work_bytes) {
+        delete c;
+        return ZZ_ERR_WORKSPACE;
+    }
+    c->arena = static_cast<unsigned char*>(d_arena);
+    c->work = static_cast<unsigned char*>(d_workspace);
+    c->kind.resize((size_t)c->L * c->Hkv);
+    c->nR.assign(c->L, 0);
+    c->heads.resize((size_t)c->L * c->Hkv);
+    c->has_mixed = false;
+    for (int l = 0; l < c->L; ++l) {
+        int r = 0;
+        for (int h = 0; h < c->Hkv; ++h) {
+            c->kind[(size_t)l * c->Hkv + h] = kind_of(cfg, l, h);
+            r += c->kind[(size_t)l * c->Hkv + h];
+        }
+        c->nR[l] = r;
+        int ir = 0, is = r;
+        for (int h = 0; h < c->Hkv; ++h) {
+            if (c->kind[(size_t)l * c->Hkv + h]) c->heads[(size_t)l * c->Hkv + ir++] = h;
+            else c->heads[(size_t)l * c->Hkv + is++] = h;
+        }
+        if (r > 0 && r < c->Hkv) c->has_mixed = true;
+    }
+    c->cap.assign(cfg->capacity, cfg->capacity + c->B);
+    c->len.assign((size_t)c->L * c->B, 0);
+
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = zz::decode_setup();
+    if (e == cudaSuccess) e = zz::prefill_setup();
+    if (e == cudaSuccess) e = cudaMemset(c->arena, 0, c->lay.arena_bytes);
+    if (e == cudaSuccess) e = cudaMemset(c->work, 0, c->lay.off_part_ml);
+    if (e == cudaSuccess) e = cudaMemset(c->work + c->lay.off_pos, 0xff, (size_t)c->L * c->B * c->ring * sizeof(int));
+    if (e == cudaSuccess)
+        e = cudaMemcpy(c->work + c->lay.off_desc, c->desc.data(), c->desc.size() * sizeof(SeqDesc),
+                       cudaMemcpyHostToDevice);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(c->work + c->lay.off_heads, c->heads.data(), c->heads.size() * sizeof(int),
+                       cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        delete c;
+        return ZZ_ERR_CUDA;
+    }
+    c->have_tmap_arena = encode_rows2d(&c->tmap_arena, c->arena, (long long)(c->lay.arena_bytes / (kD * 2)));
+    *out = c;
+    return ZZ_OK;
+}
+
+int zz_cache_destroy(zz_cache_t* c) {
+    if (!c) return ZZ_ERR_INVALID_ARG;
+    delete c;
+    return ZZ_OK;
+}
+
+int zz_cache_reset(zz_cache_t* c, int seq, void* stream) {
+    if (!c || seq < -1 || seq >= c->B) return ZZ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (zz::launch_reset(c->d_len(0), c->d_pos(0), c->L, c->B, c->ring, seq, st) != cudaSuccess)
+        return ZZ_ERR_CUDA;
+    for (int l = 0; l < c->L; ++l)
+        for (int b = 0; b < c->B; ++b)
+            if (seq < 0 || seq == b) c->len[(size_t)l * c->B + b] = 0;
+    return ZZ_OK;
+}
+
+int zz_cache_len(const zz_cache_t* c, int layer, int seq, int32_t* len) {
+    if (bad_layer(c, layer) || seq < 0 || seq >= c->B || !len) return ZZ_ERR_INVALID_ARG;
+    *len = c->len[(size_t)layer * c->B + seq];
+    return ZZ_OK;
+}
+
+int zz_tune(zz_cache_t* c, const char* key, int value) {
+    if (!c || !key) return ZZ_ERR_INVALID_ARG;
+    if (!strcmp(key, "decode_min_chunk")) {
+        if (value < 16 || value % 16) return ZZ_ERR_INVALID_ARG;
+        c->decode_min_chunk = value;
+        return ZZ_OK;
+    }
+    return ZZ_ERR_INVALID_ARG;
+}
+
+int zz_kv_append(zz_cache_t* c, int layer, const void* d_k, const void* d_v, const int32_t* h_n_new,
+                 void* stream) {
+    if (bad_layer(c, layer) || !d_k || !d_v || !h_n_new) return ZZ_ERR_INVALID_ARG;
+    if (((uintptr_t)d_k | (uintptr_t)d_v) & 15) return ZZ_ERR_INVALID_ARG;
+    const int nR = c->nR[layer], nS = c->Hkv - nR;
+    long long total = 0, worst = 0;
+    for (int b = 0; b < c->B; ++b) {
+        if (h_n_new[b] < 0) return ZZ_ERR_INVALID_ARG;
+        const long long nl = (long long)c->len[(size_t)layer * c->B + b] + h_n_new[b];
+        if (nl > 0x7fffffffLL) return ZZ_ERR_CAPACITY;
+        if (nR > 0 && nl > c->cap[b]) return ZZ_ERR_CAPACITY;
+        total += h_n_new[b];
+    }
+    if (total == 0) return ZZ_OK;
+    zz::AppendParams p;
+    memset(&p, 0, sizeof p);
+    p.arena = c->d_arena();
+    p.desc = c->d_desc(layer);
+    p.len = c->d_len(layer);
+    p.pos = c->d_pos(layer);
+    p.counter = c->d_append_counter();
+    p.k_new = static_cast<const __nv_bfloat16*>(d_k);
+    p.v_new = static_cast<const __nv_bfloat16*>(d_v);
+    p.head_list = c->d_heads(layer);
+    p.nR = nR; p.Hkv = c->Hkv; p.ring = c->ring; p.S = c->S; p.W = c->W; p.B = c->B;
+    int off = 0;
+    for (int b = 0; b < c->B; ++b) {
+        p.n_new[b] = h_n_new[b];
+        p.tok_off[b] = off;
+        off += h_n_new[b];
+        const long long cand = h_n_new[b] < c->ring ? h_n_new[b] : c->ring;
+        const long long work = ((long long)h_n_new[b] * nR + cand * nS) * 16;
+        if (work > worst) worst = work;
+    }
+    const long long gx = (worst + 255) / 256;
+    if (gx > 0x7fffffffLL) return ZZ_ERR_UNSUPPORTED;
+    if (zz::launch_append(p, (int)gx, static_cast<cudaStream_t>(stream)) != cudaSuccess) return ZZ_ERR_CUDA;
+    for (int b = 0; b < c->B; ++b) c->len[(size_t)layer * c->B + b] += h_n_new[b];
+    return ZZ_OK;
+}
+
+int zz_decode_attn(zz_cache_t* c, int layer, const void* d_q, void* d_out, void* stream) {
+    if (bad_layer(c, layer) || !d_q || !d_out) return ZZ_ERR_INVALID_ARG;
+    if (((uintptr_t)d_q | (uintptr_t)d_out) & 15) return ZZ_ERR_INVALID_ARG;
+    for (int b = 0; b < c->B; ++b)
+        if (c->len[(size_t)layer * c->B + b] < 1) return ZZ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(d_q);
+    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(d_out);
+    if (!c->mixed(layer)) {
+        const int kind = c->nR[layer] ? ZZ_KIND_RETRIEVAL : ZZ_KIND_STREAMING;
+        return launch_decode_group(c, layer, kind, q, out, 0, st);
+    }
+    // DuoAttention-style layer: gather the heads of each kind, one pass per kind, scatter back
+    int r = regroup(c, layer, q, c->d_qc(), c->B, 1, st);
+    if (r == ZZ_OK) r = launch_decode_group(c, layer, ZZ_KIND_RETRIEVAL, c->d_qc(), c->d_oc(), 0, st);
+    if (r == ZZ_OK)
+        r = launch_decode_group(c, layer, ZZ_KIND_STREAMING, c->d_qc(), c->d_oc(), c->nR[layer] * c->G, st);
+    if (r == ZZ_OK) r = regroup(c, layer, c->d_oc(), out, c->B, 0, st);
+    return r;
+}
+
+int zz_decode_step(zz_cache_t* c, int layer, const void* d_q, const void* d_k, const void* d_v, void* d_out,
+                   void* stream) {
+    if (bad_layer(c, layer)) return ZZ_ERR_INVALID_ARG;
+    int32_t ones[ZZ_MAX_BATCH];
+    for (int b = 0; b < c->B; ++b) ones[b] = 1;
+    if (!d_q || !d_out) return ZZ_ERR_INVALID_ARG;
+    const int r = zz_kv_append(c, layer, d_k, d_v, ones, stream);
+    if (r != ZZ_OK) return r;
+    return zz_decode_attn(c, layer, d_q, d_out, stream);
+}
+
+int zz_prefill_attn(zz_cache_t* c, int layer, const void* d_q, const void* d_k, const void* d_v, void* d_out,
+                    const int32_t* h_n_new, void* stream) {
+    if (bad_layer(c, layer) || !d_q || !d_k || !d_v || !d_out || !h_n_new) return ZZ_ERR_INVALID_ARG;
+    if (((uintptr_t)d_q | (uintptr_t)d_k | (uintptr_t)d_v | (uintptr_t)d_out) & 15) return ZZ_ERR_INVALID_ARG;
+    long long total = 0;
+    for (int b = 0; b < c->B; ++b) {
+        if (h_n_new[b] < 0) return ZZ_ERR_INVALID_ARG;
+        if ((long long)c->len[(size_t)layer * c->B + b] + h_n_new[b] > 0x7fffffffLL) return ZZ_ERR_CAPACITY;
+        total += h_n_new[b];
+    }
+    if (total == 0) return ZZ_OK;
+    if (!c->have_tmap_arena) return ZZ_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(d_q);
+    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(d_out);
+    alignas(64) CUtensorMap tq, tk, tv;
+    if (!encode_rows3d(&tk, d_k, total, c->Hkv) || !encode_rows3d(&tv, d_v, total, c->Hkv)) return ZZ_ERR_CUDA;
+    if (!c->mixed(layer)) {
+        if (!encode_rows3d(&tq, q, total, c->Hq)) return ZZ_ERR_CUDA;
+        const int kind = c->nR[layer] ? ZZ_KIND_RETRIEVAL : ZZ_KIND_STREAMING;
+        return launch_prefill_group(c, layer, kind, &tq, &tk, &tv, out, 0, h_n_new, st);
+    }
+    if (total > c->max_new) return ZZ_ERR_WORKSPACE;
+    if (!encode_rows3d(&tq, c->d_qc(), total, c->Hq)) return ZZ_ERR_CUDA;
+    int r = regroup(c, layer, q, c->d_qc(), total, 1, st);
+    if (r == ZZ_OK) r = launch_prefill_group(c, layer, ZZ_KIND_RETRIEVAL, &tq, &tk, &tv, c->d_oc(), 0, h_n_new, st);
+    if (r == ZZ_OK)
+        r = launch_prefill_group(c, layer, ZZ_KIND_STREAMING, &tq, &tk, &tv, c->d_oc(), c->nR[layer] * c->G,
+                                 h_n_new, st);
+    if (r == ZZ_OK) r = regroup(c, layer, c->d_oc(), out, total, 0, st);
+    return r;
+}
+
+size_t zz_stage_bytes(const zz_cache_t* c, int64_t n_tokens) {
+    if (!c || n_tokens < 0) return 0;
+    const size_t qb = align_up((size_t)n_tokens * c->Hq * kD * 2);
+    const size_t kb = align_up((size_t)n_tokens * c->Hkv * kD * 2);
+    return 2 * qb + 2 * kb;
+}
+
+static int run_host(zz_cache_t* c, int layer, const void* h_q, const void* h_k, const void* h_v, void* h_out,
+                    const int32_t* n_new, void* d_stage, size_t stage_bytes, void* stream, bool decode) {
+    if (bad_layer(c, layer) || !h_q || !h_k || !h_v || !h_out || !d_stage || !n_new) return ZZ_ERR_INVALID_ARG;
+    long long total = 0;
+    for (int b = 0; b < c->B; ++b) {
+        if (n_new[b] < 0) return ZZ_ERR_INVALID_ARG;
+        total += n_new[b];
+    }
+    if (stage_bytes < zz_stage_bytes(c, total)) return ZZ_ERR_WORKSPACE;
+    if ((uintptr_t)d_stage % kAlign) return ZZ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t qbytes = (size_t)total * c->Hq * kD * 2, kbytes = (size_t)total * c->Hkv * kD * 2;
+    const size_t qb = align_up(qbytes), kb = align_up(kbytes);
+    unsigned char* s = static_cast<unsigned char*>(d_stage);
+    void* dq = s; void* dk = s + qb; void* dv = s + qb + kb; void* dout = s + qb + 2 * kb;
+    if (total == 0) return ZZ_OK;
+    if (cudaMemcpyAsync(dq, h_q, qbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    if (cudaMemcpyAsync(dk, h_k, kbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    if (cudaMemcpyAsync(dv, h_v, kbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    int r;
+    if (decode) {
+        r = zz_decode_step(c, layer, dq, dk, dv, dout, stream);
+    } else {
+        r = zz_prefill_attn(c, layer, dq, dk, dv, dout, n_new, stream);
+        if (r == ZZ_OK) r = zz_kv_append(c, layer, dk, dv, n_new, stream);
+    }
+    if (r != ZZ_OK) return r;
+    if (cudaMemcpyAsync(h_out, dout, qbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    return ZZ_OK;
+}
+
+int zz_decode_step_host(zz_cache_t* c, int layer, const void* h_q, const void* h_k, const void* h_v,
+                        void* h_out, void* d_stage, size_t stage_bytes, void* stream) {
+    if (!c) return ZZ_ERR_INVALID_ARG;
+    int32_t ones[ZZ_MAX_BATCH];
+    for (int b = 0; b < c->B; ++b) ones[b] = 1;
+    return run_host(c, layer, h_q, h_k, h_v, h_out, ones, d_stage, stage_bytes, stream, true);
+}
+
+int zz_prefill_host(zz_cache_t* c, int layer, const void* h_q, const void* h_k, const void* h_v, void* h_out,
+                    const int32_t* h_n_new, void* d_stage, size_t stage_bytes, void* stream) {
+    return run_host(c, layer, h_q, h_k, h_v, h_out, h_n_new, d_stage, stage_bytes, stream, false);
+}
+
+int zz_cache_export_shape(const zz_cache_t* c, int layer, int seq, int kind, int32_t* n_heads,
+                          int32_t* n_slots) {
+    if (bad_layer(c, layer) || seq < 0 || seq >= c->B || (kind != 0 && kind != 1) || !n_heads || !n_slots)
+        return ZZ_ERR_INVALID_ARG;
+    *n_heads = (kind == ZZ_KIND_RETRIEVAL) ? c->nR[layer] : c->Hkv - c->nR[layer];
+    *n_slots = (kind == ZZ_KIND_RETRIEVAL) ? c->cap[seq] : c->ring;
+    return ZZ_OK;
+}
+
+int zz_cache_export(zz_cache_t* c, int layer, int seq, int kind, void* h_k, void* h_v, int32_t* h_pos,
+                    int32_t* h_len, void* stream) {
+    int32_t nh, ns;
+    const int r = zz_cache_export_shape(c, layer, seq, kind, &nh, &ns);
+    if (r != ZZ_OK) return r;
+    if (!h_k || !h_v || !h_pos || !h_len) return ZZ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const SeqDesc& d = c->desc[(size_t)layer * c->B + seq];
+    const size_t bytes = (size_t)nh * ns * kD * 2;
+    cudaError_t e = cudaSuccess;
+    if (bytes) {
+        e = cudaMemcpyAsync(h_k, c->d_arena() + d.k_off[kind], bytes, cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(h_v, c->d_arena() + d.v_off[kind], bytes, cudaMemcpyDeviceToHost, st);
+    }
+    int dev_len = 0;
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&dev_len, c->d_len(layer) + seq, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && kind == ZZ_KIND_STREAMING)
+        e = cudaMemcpyAsync(h_pos, c->d_pos(layer) + (size_t)seq * c->ring, (size_t)c->ring * sizeof(int),
+                            cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return ZZ_ERR_CUDA;
+    *h_len = dev_len;
+    if (kind == ZZ_KIND_RETRIEVAL)
+        for (int i = 0; i < ns; ++i) h_pos[i] = (i < dev_len) ? i : -1;
+    return ZZ_OK;
+}
+
+int zz_cache_import(zz_cache_t* c, int layer, int seq, int kind, const void* h_k, const void* h_v,
+                    const int32_t* h_pos, int32_t len, void* stream) {
+    int32_t nh, ns;
+    const int r = zz_cache_export_shape(c, layer, seq, kind, &nh, &ns);
+    if (r != ZZ_OK) return r;
+    if (!h_k || !h_v || !h_pos || len < 0) return ZZ_ERR_INVALID_ARG;
+    if (kind == ZZ_KIND_RETRIEVAL && len > ns) return ZZ_ERR_CAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const SeqDesc& d = c->desc[(size_t)layer * c->B + seq];
+    const size_t bytes = (size_t)nh * ns * kD * 2;
+    cudaError_t e = cudaSuccess;
+    if (bytes) {
+        e = cudaMemcpyAsync(c->d_arena() + d.k_off[kind], h_k, bytes, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(c->d_arena() + d.v_off[kind], h_v, bytes, cudaMemcpyHostToDevice, st);
+    }
+    if (e == cudaSuccess && kind == ZZ_KIND_STREAMING)
+        e = cudaMemcpyAsync(c->d_pos(layer) + (size_t)seq * c->ring, h_pos, (size_t)c->ring * sizeof(int),
+                            cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(c->d_len(layer) + seq, &len, sizeof(int), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return ZZ_ERR_CUDA;
+    c->len[(size_t)layer * c->B + seq] = len;
+    return ZZ_OK;
+}
+
+int zz_get_last_status(zz_cache_t* c, void* stream) {
+    if (!c) return ZZ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int v = 0;
+    if (cudaMemcpyAsync(&v, c->d_status(), sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ZZ_ERR_CUDA;
+    if (v != 0) {
+        if (cudaMemsetAsync(c->d_status(), 0, sizeof(int), st) != cudaSuccess) return ZZ_ERR_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return ZZ_ERR_CUDA;
+    }
+    return v;
+}
+
+}  // extern "C"

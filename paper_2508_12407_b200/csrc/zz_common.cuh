@@ -1,0 +1,106 @@
+// Shared declarations of the CUDA path: parameter blocks passed from the host
+// dispatcher to the kernels, and small device helpers.  sm_100a only.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "zigzag.h"
+
+namespace zz {
+
+constexpr int kD = 128;            // head_dim
+constexpr int kRowBytes = kD * 2;  // one K or V row of one head
+
+// Where the stores of one (layer, sequence) live in the arena, in bf16 elements from the
+// arena base.  Index [ZZ_KIND_STREAMING] is the ring group, [ZZ_KIND_RETRIEVAL] the
+// append-only group; each group is laid out [head_in_group][slot][128].
+struct SeqDesc {
+    long long k_off[2];
+    long long v_off[2];
+    int cap;   // slots per head of the retrieval group (capacity of this sequence)
+    int pad;
+};
+
+struct AppendParams {
+    __nv_bfloat16* arena;
+    const SeqDesc* desc;     // [B] of this layer
+    int* len;                // [B] of this layer (device lengths)
+    int* pos;                // [B][ring] of this layer
+    unsigned int* counter;   // blocks-done counter (0 between launches)
+    const __nv_bfloat16* k_new;  // [sum n_new][Hkv][128]
+    const __nv_bfloat16* v_new;
+    const int* head_list;    // [Hkv] source KV heads: first nR retrieval heads, then streaming
+    int nR, Hkv, ring, S, W, B;
+    int n_new[ZZ_MAX_BATCH];
+    int tok_off[ZZ_MAX_BATCH];
+};
+
+struct DecodeParams {
+    const __nv_bfloat16* arena;
+    const SeqDesc* desc;     // [B]
+    const int* len;          // [B]
+    const __nv_bfloat16* q;  // row of sequence b, head h at q + b*q_tok_stride + (q_head0 + h)*128
+    __nv_bfloat16* out;      // same addressing as q
+    long long q_tok_stride;  // elements between consecutive sequences' rows (n_q_heads * 128)
+    int q_head0;             // first query head of this group inside a row
+    float* part_o;           // [B*Hg][max_splits][G][128]
+    float* part_ml;          // [B*Hg][max_splits][G][2]
+    unsigned int* counters;  // [B*Hg], 0 between launches
+    int* status;
+    int kind;                // which group of the layer
+    int ring;                // S+W
+    int Hg, G, B;
+    int chunk;               // tokens per split (multiple of 16)
+    int max_splits;
+    float scale_log2;        // softmax_scale * log2(e)
+    int split_start[ZZ_MAX_BATCH + 1];  // prefix sum of per-sequence split counts
+};
+
+struct GatherParams {
+    // copies rows of heads between the model's head order and the two compact group buffers
+    const __nv_bfloat16* src;
+    __nv_bfloat16* dst;
+    const int* head_list;    // [Hkv] group-ordered KV heads
+    int Hkv, G;
+    long long tokens;
+    int to_compact;          // 1: model order -> compact (gather); 0: compact -> model order (scatter)
+};
+
+struct PrefillParams {
+    const SeqDesc* desc;     // [B] of this layer
+    const int* len;          // [B] device lengths (tokens already in the store)
+    const int* pos;          // [B][ring] ring positions of this layer
+    __nv_bfloat16* out;      // row of packed token i, head h at out + i*tok_stride + (q_head0+h)*128
+    long long tok_stride;    // n_q_heads * 128
+    long long arena_row0;    // unused by the kernel (rows are derived from desc offsets)
+    const int* head_list;    // [Hkv] group-ordered source KV heads (for the chunk K/V)
+    int* status;
+    int kind;                // group served by this launch
+    int kv_head0;            // first entry of head_list that belongs to the group
+    int q_head0;             // first query head of the group inside a q/out row
+    int n_kv_total;          // KV heads per row of the chunk K/V
+    int ring, S, W, Hg, G, B;
+    int total_tiles;         // 128-row query tiles over the whole batch
+    float scale_log2;
+    int n_new[ZZ_MAX_BATCH];
+    int tok_off[ZZ_MAX_BATCH];
+    int tile_start[ZZ_MAX_BATCH + 1];
+};
+
+// ---- launchers (defined in the .cu files) -------------------------------------------
+cudaError_t launch_append(const AppendParams& p, int grid_x, cudaStream_t s);
+cudaError_t launch_decode(const DecodeParams& p, int n_items, cudaStream_t s);
+cudaError_t launch_regroup(const GatherParams& p, cudaStream_t s);
+cudaError_t launch_reset(int* len, int* pos, int L, int B, int ring, int seq, cudaStream_t s);
+cudaError_t decode_setup();
+cudaError_t prefill_setup();
+// tensor maps: q [tokens][heads][128] (3-D), chunk k and v [tokens][kv heads][128] (3-D), and the
+// arena seen as rows of 128 bf16 (2-D); opaque 128-byte CUtensorMap objects
+cudaError_t launch_prefill(const PrefillParams& p, const void* tmap_q, const void* tmap_k,
+                           const void* tmap_v, const void* tmap_arena, int n_items, cudaStream_t s);
+
+void count_launch(int n = 1);
+
+}  // namespace zz

@@ -1,0 +1,351 @@
+// Decode attention: one query token per sequence over a KV store.
+//
+// The same kernel serves retrieval layers (split-sequence flash decoding over the whole
+// append-only store) and streaming layers (a single pass over the occupied ring slots in
+// physical order: after an append the ring holds exactly the visible set, and the occupied
+// slots are always the first min(len, S+W) ones).
+//
+// Work item = (sequence, KV head of the group, token range).  The G query heads that share a
+// KV head are the rows of one 16-row MMA tile, so every K/V byte is read from HBM once and
+// used by all of them.  Each warp streams its own 16-token blocks through a private
+// multi-stage cp.async pipeline (16-byte coalesced loads, zero-filled past the range end),
+// keeps a private online-softmax state, and the warps, then the splits, are merged with the
+// usual (max, sum, weighted output) rule.  The last CTA of a (sequence, head) to finish does
+// the split merge, so there is no second launch.
+//
+// The roofline of this kernel is HBM bandwidth: 2 * 128 * 2 bytes per token and KV head.
+#include "zz_common.cuh"
+
+namespace zz {
+
+namespace {
+
+constexpr int kWarps = 4;
+constexpr int kBlk = 16;                       // tokens per warp step
+constexpr int kStages = 3;
+constexpr int kStageBytes = kBlk * kRowBytes;  // 4 KiB of K (and as much of V) per stage
+constexpr int kWarpSmem = kStages * 2 * kStageBytes;
+constexpr int kSmemBytes = kWarps * kWarpSmem;  // 96 KiB -> two CTAs per SM
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
+                                            uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1,
+                                                  uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                         uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};\n"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Issue the loads of one 16-token block (K and V rows of one head) into a stage.
+// Row r, 16-byte piece c lands at r*256 + ((c ^ (r & 7)) * 16): conflict-free for ldmatrix.
+__device__ __forceinline__ void load_block(uint32_t stage_k, uint32_t stage_v, const __nv_bfloat16* kbase,
+                                           const __nv_bfloat16* vbase, int tok0, int tok_end, int lane) {
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+        const int idx = it * 32 + lane;
+        const int r = idx >> 4, c = idx & 15;
+        const int tok = tok0 + r;
+        const int ok = tok < tok_end;
+        const long long off = (long long)(ok ? tok : tok0) * kD + c * 8;
+        const uint32_t so = r * kRowBytes + ((c ^ (r & 7)) << 4);
+        cp_async16(stage_k + so, kbase + off, ok ? 16 : 0);
+        cp_async16(stage_v + so, vbase + off, ok ? 16 : 0);
+    }
+}
+
+// HI = group size above 8 (rows 8..15 of the tile carry query heads too).
+template <bool HI>
+__global__ void __launch_bounds__(kWarps * 32, 2) decode_kernel(const DecodeParams p) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    __shared__ int s_is_last;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int grp = lane >> 2, tig = lane & 3;
+
+    // ---- which work item -----------------------------------------------------------
+    const int item = blockIdx.x;
+    int b = 0;
+    while (b + 1 < p.B && item >= p.split_start[b + 1] * p.Hg) ++b;
+    const int local = item - p.split_start[b] * p.Hg;
+    const int hg = local % p.Hg;
+    const int split = local / p.Hg;
+    const int nsplit = p.split_start[b + 1] - p.split_start[b];
+
+    const SeqDesc sd = p.desc[b];
+    const int len = p.len[b];
+    const int n = (p.kind == ZZ_KIND_RETRIEVAL) ? len : min(len, p.ring);
+    const long long slots_per_head = (p.kind == ZZ_KIND_RETRIEVAL) ? sd.cap : p.ring;
+    const __nv_bfloat16* kbase = p.arena + sd.k_off[p.kind] + (long long)hg * slots_per_head * kD;
+    const __nv_bfloat16* vbase = p.arena + sd.v_off[p.kind] + (long long)hg * slots_per_head * kD;
+
+    const int s0 = min(split * p.chunk, n);
+    const int s1 = (split == nsplit - 1) ? n : min(n, s0 + p.chunk);
+    const int nblk = (s1 - s0 + kBlk - 1) / kBlk;              // 16-token blocks of this CTA
+    const int my_blocks = (nblk > warp) ? (nblk - warp + kWarps - 1) / kWarps : 0;
+
+    // ---- query fragments: rows = the G heads of this KV head ---------------------------
+    const int G = p.G;
+    const __nv_bfloat16* qb = p.q + ((long long)b * p.q_tok_stride) + (long long)(p.q_head0 + hg * G) * kD;
+    uint32_t qa[8][4];
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) {
+        const int d0 = kk * 16 + tig * 2;
+        qa[kk][0] = (grp < G) ? *reinterpret_cast<const uint32_t*>(qb + grp * kD + d0) : 0u;
+        qa[kk][2] = (grp < G) ? *reinterpret_cast<const uint32_t*>(qb + grp * kD + d0 + 8) : 0u;
+        if (HI) {
+            qa[kk][1] = (grp + 8 < G) ? *reinterpret_cast<const uint32_t*>(qb + (grp + 8) * kD + d0) : 0u;
+            qa[kk][3] = (grp + 8 < G) ? *reinterpret_cast<const uint32_t*>(qb + (grp + 8) * kD + d0 + 8) : 0u;
+        } else {
+            qa[kk][1] = 0u;
+            qa[kk][3] = 0u;
+        }
+    }
+
+    // ---- per-warp state ------------------------------------------------------------------
+    constexpr int NR = HI ? 2 : 1;       // row halves carried
+    float o[16][4];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+    float m_run[2] = {-INFINITY, -INFINITY};
+    float l_run[2] = {0.f, 0.f};
+
+    const uint32_t wbase = smem_u32(smem) + warp * kWarpSmem;
+
+    // prologue: fill kStages-1 stages
+#pragma unroll
+    for (int s = 0; s < kStages - 1; ++s) {
+        if (s < my_blocks) {
+            const int tok0 = s0 + (warp + s * kWarps) * kBlk;
+            load_block(wbase + s * 2 * kStageBytes, wbase + s * 2 * kStageBytes + kStageBytes, kbase, vbase,
+                       tok0, s1, lane);
+        }
+        cp_async_commit();
+    }
+
+    for (int it = 0; it < my_blocks; ++it) {
+        {   // keep the pipeline full
+            const int nx = it + kStages - 1;
+            if (nx < my_blocks) {
+                const int st = nx % kStages;
+                const int tok0 = s0 + (warp + nx * kWarps) * kBlk;
+                load_block(wbase + st * 2 * kStageBytes, wbase + st * 2 * kStageBytes + kStageBytes, kbase,
+                           vbase, tok0, s1, lane);
+            }
+            cp_async_commit();
+        }
+        cp_async_wait<kStages - 1>();
+        __syncwarp();
+
+        const int st = it % kStages;
+        const uint32_t sk = wbase + st * 2 * kStageBytes;
+        const uint32_t sv = sk + kStageBytes;
+        const int tok0 = s0 + (warp + it * kWarps) * kBlk;
+
+        // S = Q K^T for 16 tokens: two 8-token column tiles
+        float sc[2][4];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) { sc[i][0] = sc[i][1] = sc[i][2] = sc[i][3] = 0.f; }
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+            const int r = (lane & 7) + ((lane >> 4) << 3);
+            const int c = kk * 2 + ((lane >> 3) & 1);
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4(sk + r * kRowBytes + ((c ^ (r & 7)) << 4), b0, b1, b2, b3);
+            mma_bf16(sc[0], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b0, b1);
+            mma_bf16(sc[1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b2, b3);
+        }
+
+        // online softmax in the log2 domain; mask tokens past the range end
+        const int valid = s1 - tok0;   // >= 1
+        uint32_t pa[4];
+#pragma unroll
+        for (int hf = 0; hf < NR; ++hf) {
+            float t[4];
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int col = nt * 8 + tig * 2 + e;
+                    const float x = sc[nt][hf * 2 + e] * p.scale_log2;
+                    t[nt * 2 + e] = (col < valid) ? x : -INFINITY;
+                }
+            }
+            float mx = fmaxf(fmaxf(t[0], t[1]), fmaxf(t[2], t[3]));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float m_new = fmaxf(m_run[hf], mx);      // finite: column 0 is always valid
+            const float alpha = fast_exp2(m_run[hf] - m_new);  // 0 on the first block
+            float ps = 0.f;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                t[e] = fast_exp2(t[e] - m_new);
+                ps += t[e];
+            }
+            l_run[hf] = l_run[hf] * alpha + ps;
+            m_run[hf] = m_new;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                o[i][hf * 2 + 0] *= alpha;
+                o[i][hf * 2 + 1] *= alpha;
+            }
+            pa[hf] = pack_bf16(t[0], t[1]);          // tokens 0..7 of the block  (k low)
+            pa[2 + hf] = pack_bf16(t[2], t[3]);      // tokens 8..15              (k high)
+        }
+        if (!HI) { pa[1] = 0u; pa[3] = 0u; }
+
+        // O += P V
+#pragma unroll
+        for (int nn = 0; nn < 8; ++nn) {
+            const int r = (lane & 7) + (((lane >> 3) & 1) << 3);
+            const int c = nn * 2 + (lane >> 4);
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4_trans(sv + r * kRowBytes + ((c ^ (r & 7)) << 4), b0, b1, b2, b3);
+            mma_bf16(o[2 * nn], pa[0], pa[1], pa[2], pa[3], b0, b1);
+            mma_bf16(o[2 * nn + 1], pa[0], pa[1], pa[2], pa[3], b2, b3);
+        }
+        __syncwarp();
+    }
+    cp_async_wait<0>();
+
+    // ---- merge the warps of this CTA ---------------------------------------------------------
+#pragma unroll
+    for (int hf = 0; hf < NR; ++hf) {
+        l_run[hf] += __shfl_xor_sync(0xffffffffu, l_run[hf], 1);
+        l_run[hf] += __shfl_xor_sync(0xffffffffu, l_run[hf], 2);
+    }
+    __syncthreads();   // every warp is done with its pipeline memory
+    float* sm_o = reinterpret_cast<float*>(smem);                  // [kWarps][16][128]
+    float* sm_ml = sm_o + kWarps * 16 * kD;                        // [kWarps][16][2]
+#pragma unroll
+    for (int hf = 0; hf < NR; ++hf) {
+        const int row = grp + hf * 8;
+        if (row < G) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                float2 v2 = make_float2(o[i][hf * 2], o[i][hf * 2 + 1]);
+                *reinterpret_cast<float2*>(sm_o + (warp * 16 + row) * kD + i * 8 + tig * 2) = v2;
+            }
+            if (tig == 0) {
+                sm_ml[(warp * 16 + row) * 2 + 0] = m_run[hf];
+                sm_ml[(warp * 16 + row) * 2 + 1] = l_run[hf];
+            }
+        }
+    }
+    __syncthreads();
+
+    const int d = threadIdx.x;   // 128 threads = 128 output dims
+    const long long pair = (long long)b * p.Hg + hg;
+    __nv_bfloat16* outb = p.out + ((long long)b * p.q_tok_stride) + (long long)(p.q_head0 + hg * G) * kD;
+    for (int row = 0; row < G; ++row) {
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) M = fmaxf(M, sm_ml[(w * 16 + row) * 2]);
+        float L = 0.f, acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            const float mw = sm_ml[(w * 16 + row) * 2];
+            const float f = (mw == -INFINITY) ? 0.f : fast_exp2(mw - M);
+            L += f * sm_ml[(w * 16 + row) * 2 + 1];
+            acc += f * sm_o[(w * 16 + row) * kD + d];
+        }
+        if (nsplit == 1) {
+            outb[row * kD + d] = __float2bfloat16_rn(acc / L);
+        } else {
+            const long long po = ((pair * p.max_splits + split) * G + row);
+            p.part_o[po * kD + d] = acc;
+            if (d == 0) {
+                p.part_ml[po * 2 + 0] = M;
+                p.part_ml[po * 2 + 1] = L;
+            }
+        }
+    }
+    if (nsplit == 1) return;
+
+    // ---- last CTA of this (sequence, head) merges the splits -----------------------------------
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int prev = atomicAdd(p.counters + pair, 1u);
+        s_is_last = (prev == (unsigned int)(nsplit - 1));
+    }
+    __syncthreads();
+    if (!s_is_last) return;
+    __threadfence();
+    for (int row = 0; row < G; ++row) {
+        float M = -INFINITY;
+        for (int s = 0; s < nsplit; ++s) {
+            const long long po = ((pair * p.max_splits + s) * G + row);
+            M = fmaxf(M, __ldcg(p.part_ml + po * 2));
+        }
+        float L = 0.f, acc = 0.f;
+        for (int s = 0; s < nsplit; ++s) {
+            const long long po = ((pair * p.max_splits + s) * G + row);
+            const float ms = __ldcg(p.part_ml + po * 2);
+            const float f = (ms == -INFINITY) ? 0.f : fast_exp2(ms - M);
+            L += f * __ldcg(p.part_ml + po * 2 + 1);
+            acc += f * __ldcg(p.part_o + po * kD + d);
+        }
+        outb[row * kD + d] = __float2bfloat16_rn(acc / L);
+    }
+    if (threadIdx.x == 0) p.counters[pair] = 0u;
+}
+
+}  // namespace
+
+cudaError_t decode_setup() {
+    cudaError_t e = cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+}
+
+cudaError_t launch_decode(const DecodeParams& p, int n_items, cudaStream_t s) {
+    if (n_items <= 0) return cudaSuccess;
+    if (p.G > 8)
+        decode_kernel<true><<<n_items, kWarps * 32, kSmemBytes, s>>>(p);
+    else
+        decode_kernel<false><<<n_items, kWarps * 32, kSmemBytes, s>>>(p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace zz

@@ -1,0 +1,97 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol
+the header declares, and validates configurations without touching a device."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2508_12407_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "zigzag.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load()
+
+
+def declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(zz_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_symbols_exported(lib):
+    names = declared_functions()
+    assert len(names) >= 18
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in zigzag.h but not exported"
+        assert n in binding.SYMBOLS, f"{n} has no binding"
+
+
+def test_version_and_status_strings(lib):
+    assert binding.version() >= 100
+    seen = set()
+    for code in [0, -1, -2, -3, -4, -5, -6]:
+        s = binding.status_str(code)
+        assert s and s != "unknown status" and s not in seen
+        seen.add(s)
+    assert binding.status_str(-99) == "unknown status"
+
+
+def make_cfg(**kw):
+    L, B = kw.get("L", 2), kw.get("B", 1)
+    kinds = np.array(kw.get("kinds", [1, 0]), dtype=np.uint8)
+    cap = np.array(kw.get("cap", [1024] * B), dtype=np.int32)
+    cfg = binding.ZZConfig(L, B, kw.get("Hq", 8), kw.get("Hkv", 2), kw.get("D", 128), kw.get("S", 64),
+                           kw.get("W", 256), kw.get("max_new", 2048), kw.get("scale", 0.088),
+                           kinds.ctypes.data, None, cap.ctypes.data)
+    cfg._keep = (kinds, cap)
+    return cfg
+
+
+def query(lib, cfg):
+    a, w = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    rc = lib.zz_cache_query(ctypes.byref(cfg), ctypes.byref(a), ctypes.byref(w))
+    return rc, a.value, w.value
+
+
+def test_query_sizes(lib):
+    rc, a, w = query(lib, make_cfg())
+    assert rc == 0
+    # layer 0 retrieval: 2 heads * 1024 slots * 128 * 2 B for K and for V; layer 1: ring of 320 slots
+    expect = 2 * (2 * 1024 * 256) + 2 * (2 * 320 * 256)
+    assert expect <= a <= expect + 128 * 256 + 256
+    assert w > 0 and a % 256 == 0 and w % 256 == 0
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(D=64), binding.ZZ_ERR_UNSUPPORTED),
+    (dict(Hq=6, Hkv=4), binding.ZZ_ERR_UNSUPPORTED),
+    (dict(Hq=34, Hkv=2), binding.ZZ_ERR_UNSUPPORTED),
+    (dict(B=65, cap=[8] * 65, max_new=100), binding.ZZ_ERR_UNSUPPORTED),
+    (dict(W=0), binding.ZZ_ERR_INVALID_ARG),
+    (dict(S=-1), binding.ZZ_ERR_INVALID_ARG),
+    (dict(cap=[0]), binding.ZZ_ERR_INVALID_ARG),
+    (dict(scale=0.0), binding.ZZ_ERR_INVALID_ARG),
+    (dict(max_new=0), binding.ZZ_ERR_INVALID_ARG),
+])
+def test_query_rejects_bad_configs(lib, kw, code):
+    rc, _, _ = query(lib, make_cfg(**kw))
+    assert rc == code
+
+
+def test_null_arguments(lib):
+    assert lib.zz_cache_query(None, None, None) == binding.ZZ_ERR_INVALID_ARG
+    cfg = make_cfg()
+    assert lib.zz_cache_query(ctypes.byref(cfg), None, None) == binding.ZZ_ERR_INVALID_ARG
+    assert lib.zz_cache_destroy(None) == binding.ZZ_ERR_INVALID_ARG
+    assert lib.zz_decode_attn(None, 0, None, None, None) == binding.ZZ_ERR_INVALID_ARG
+    assert lib.zz_kv_append(None, 0, None, None, None, None) == binding.ZZ_ERR_INVALID_ARG
+    assert lib.zz_prefill_attn(None, 0, None, None, None, None, None, None) == binding.ZZ_ERR_INVALID_ARG
+    assert lib.zz_get_last_status(None, None) == binding.ZZ_ERR_INVALID_ARG
+    assert lib.zz_stage_bytes(None, 5) == 0
