@@ -26,6 +26,7 @@ constexpr int kStages = 3;
 constexpr int kStageBytes = kBlk * kRowBytes;  // 4 KiB of K (and as much of V) per stage
 constexpr int kWarpSmem = kStages * 2 * kStageBytes;
 constexpr int kSmemBytes = kWarps * kWarpSmem;  // 96 KiB -> two CTAs per SM
+constexpr int kMaxSplitsSmem = 128;             // >= the host's split limit
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return (uint32_t)__cvta_generic_to_shared(p);
@@ -310,21 +311,43 @@ __global__ void __launch_bounds__(kWarps * 32, 2) decode_kernel(const DecodePara
     __syncthreads();
     if (!s_is_last) return;
     __threadfence();
+    // (max, sum) of every split and row into shared memory, then each thread owns one output
+    // dimension and streams the partial outputs with independent loads in flight
+    float* sm_m = reinterpret_cast<float*>(smem);            // [G][nsplit]
+    float* sm_f = sm_m + 16 * kMaxSplitsSmem;                // [G][nsplit] -> scale factors
+    for (int i = threadIdx.x; i < nsplit * G; i += blockDim.x) {
+        const int s = i / G, row = i % G;
+        const long long po = ((pair * p.max_splits + s) * G + row);
+        sm_m[row * kMaxSplitsSmem + s] = __ldcg(p.part_ml + po * 2);
+        sm_f[row * kMaxSplitsSmem + s] = __ldcg(p.part_ml + po * 2 + 1);
+    }
+    __syncthreads();
     for (int row = 0; row < G; ++row) {
         float M = -INFINITY;
-        for (int s = 0; s < nsplit; ++s) {
-            const long long po = ((pair * p.max_splits + s) * G + row);
-            M = fmaxf(M, __ldcg(p.part_ml + po * 2));
+        for (int s = 0; s < nsplit; ++s) M = fmaxf(M, sm_m[row * kMaxSplitsSmem + s]);
+        float L = 0.f, acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
+        const float* po = p.part_o + ((pair * p.max_splits) * G + row) * kD + d;
+        const long long sstride = (long long)G * kD;
+        int s = 0;
+        for (; s + 4 <= nsplit; s += 4) {
+            const float v0 = __ldcg(po + (s + 0) * sstride), v1 = __ldcg(po + (s + 1) * sstride);
+            const float v2 = __ldcg(po + (s + 2) * sstride), v3 = __ldcg(po + (s + 3) * sstride);
+            float f[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float ms = sm_m[row * kMaxSplitsSmem + s + u];
+                f[u] = (ms == -INFINITY) ? 0.f : fast_exp2(ms - M);
+                L += f[u] * sm_f[row * kMaxSplitsSmem + s + u];
+            }
+            acc0 += f[0] * v0; acc1 += f[1] * v1; acc2 += f[2] * v2; acc3 += f[3] * v3;
         }
-        float L = 0.f, acc = 0.f;
-        for (int s = 0; s < nsplit; ++s) {
-            const long long po = ((pair * p.max_splits + s) * G + row);
-            const float ms = __ldcg(p.part_ml + po * 2);
+        for (; s < nsplit; ++s) {
+            const float ms = sm_m[row * kMaxSplitsSmem + s];
             const float f = (ms == -INFINITY) ? 0.f : fast_exp2(ms - M);
-            L += f * __ldcg(p.part_ml + po * 2 + 1);
-            acc += f * __ldcg(p.part_o + po * kD + d);
+            L += f * sm_f[row * kMaxSplitsSmem + s];
+            acc0 += f * __ldcg(po + s * sstride);
         }
-        outb[row * kD + d] = __float2bfloat16_rn(acc / L);
+        outb[row * kD + d] = __float2bfloat16_rn(((acc0 + acc1) + (acc2 + acc3)) / L);
     }
     if (threadIdx.x == 0) p.counters[pair] = 0u;
 }

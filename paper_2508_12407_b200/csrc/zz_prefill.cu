@@ -1,9 +1,526 @@
-// placeholder until the tcgen05 prefill kernel lands
+// Prefill attention on the 5th-generation tensor cores: tcgen05.mma with the S = Q K^T and
+// O = P V accumulators in tensor memory, operands staged in shared memory by TMA.
+//
+// One kernel serves both kinds of layer.  A retrieval head visits every KV tile up to the
+// diagonal (causal flash attention); a streaming head visits only the tiles that can hold
+// visible keys -- the sink tiles and the local band -- and applies the token-exact
+// visibility rule inside them (block sparsity is an execution strategy, not the mask).
+// Keys come from two places: the store as it stood before the call (append-only rows or
+// ring slots, positions from pos[]) and the new chunk itself.
+//
+// CTA = one 128-token query tile x two query heads of the same KV head, so each K/V tile is
+// fetched once for two score tiles and the two tiles ping-pong on the tensor pipe:
+//   warp 0      TMA producer (one elected lane)
+//   warp 1      MMA issuer   (one elected lane)
+//   warps 2-5   softmax / correction / epilogue of tile 0 (one thread per query row)
+//   warps 6-9   the same for tile 1
+// Tensor memory (512 columns): tile t has S_t at column 256 t (128 fp32 columns; the bf16
+// probabilities P_t overwrite its first 64 columns and feed the PV MMA as the A operand from
+// tensor memory) and O_t at column 256 t + 128.
+// Every mbarrier wait is bounded; when one expires the kernel records ZZ_ERR_TIMEOUT in the
+// status word, stops waiting long for anything else, frees its tensor memory and returns.
+#include <cuda.h>
+
 #include "zz_common.cuh"
+
 namespace zz {
-cudaError_t prefill_setup() { return cudaSuccess; }
-cudaError_t launch_prefill(const PrefillParams&, const void*, const void*, const void*, const void*, int,
-                           cudaStream_t) {
-    return cudaErrorNotSupported;
+
+namespace {
+
+constexpr int kTile = 128;
+constexpr int kSubBytes = 128 * 128;        // [128 rows][64 bf16] sub-tile, 128-byte swizzled
+constexpr int kTileBytes = 2 * kSubBytes;   // a full [128][128] bf16 tile
+constexpr int kStages = 4;                  // ring of K and V tiles (K_0, V_0, K_1, V_1, ...)
+constexpr int kThreads = 320;
+constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 1024;
+constexpr uint32_t kMaxPolls = 1u << 22;
+constexpr uint32_t kAbortPolls = 1u << 10;
+constexpr float kRescaleThreshold = 8.f;    // log2 units of slack before O is rescaled
+
+// instruction descriptor: fp32 accumulate, bf16 A and B, M = 128, N = 128
+constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);   // B (= V) is MN-major
+
+struct Shared {
+    uint64_t q_full;
+    uint64_t kv_full[kStages];
+    uint64_t kv_empty[kStages];
+    uint64_t s_full[2];
+    uint64_t p_full[2];
+    uint64_t o_full;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (after flagging the error) if the phase never completed.
+__device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Shared* sh, int* status) {
+    const uint32_t limit = (*(volatile int*)&sh->abort_flag) ? kAbortPolls : kMaxPolls;
+    for (uint32_t i = 0; i < limit; ++i) {
+        if (mbar_try(bar, parity)) return true;
+        if ((i & 4095u) == 4095u && (*(volatile int*)&sh->abort_flag)) break;
+    }
+    *(volatile int*)&sh->abort_flag = 1;
+    atomicExch(status, ZZ_ERR_TIMEOUT);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z,
+                                            uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
+        : "memory");
+}
+
+// shared-memory matrix descriptor, 128-byte swizzle, sm_100 descriptor version
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= 1ull << 46;
+    d |= 2ull << 61;
+    return d;
+}
+
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"((uint32_t)acc)
+        : "memory");
+}
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, bool acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"((uint32_t)acc)
+        : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 32 lanes x 32 consecutive fp32 columns: thread i of the warp gets lane (base + i)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+    uint32_t* r = reinterpret_cast<uint32_t*>(v);
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
+    const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
+          "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Which KV tiles a query tile visits, in order: store tiles, then chunk tiles (sink tiles of
+// the chunk that lie before the band, then the band up to the diagonal).
+struct TilePlan {
+    int n_store;       // tiles over the store (rows 0.. of the append-only store / ring slots)
+    int n_sink_chunk;  // leading chunk tiles visited only for their sinks
+    int band_lo;       // first chunk tile of the band
+    int n_total;
+    int n_occ;         // occupied store rows (P, or min(P, S+W))
+};
+
+__device__ __forceinline__ TilePlan make_plan(int kind, int P, int C, int qt, int S, int W, int ring) {
+    TilePlan t;
+    const int r0 = qt * kTile;
+    if (kind == ZZ_KIND_RETRIEVAL) {
+        t.n_occ = P;
+        t.n_store = (P + kTile - 1) / kTile;
+        t.n_sink_chunk = 0;
+        t.band_lo = 0;
+    } else {
+        t.n_occ = min(P, ring);
+        const int full = (t.n_occ + kTile - 1) / kTile;
+        const int sink_tiles = (min(S, t.n_occ) + kTile - 1) / kTile;
+        t.n_store = (r0 < W) ? full : sink_tiles;   // rows >= W see no recent key of the old store
+        const int n_sink_c = max(0, min(S - P, C));
+        const int ns = (n_sink_c + kTile - 1) / kTile;
+        const int lo = r0 - W + 1;
+        t.band_lo = lo > 0 ? lo / kTile : 0;
+        t.n_sink_chunk = min(ns, t.band_lo);
+    }
+    t.n_total = t.n_store + t.n_sink_chunk + (qt - t.band_lo + 1);
+    return t;
+}
+
+// tile j of the plan: from the store (is_chunk = false) or the chunk, starting at row `start`
+__device__ __forceinline__ void plan_tile(const TilePlan& t, int j, bool& is_chunk, int& start) {
+    if (j < t.n_store) {
+        is_chunk = false;
+        start = j * kTile;
+    } else {
+        is_chunk = true;
+        const int c = j - t.n_store;
+        start = (c < t.n_sink_chunk ? c : t.band_lo + (c - t.n_sink_chunk)) * kTile;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q,
+               const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
+               const __grid_constant__ CUtensorMap tmap_arena) {
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ Shared sh;
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sm_q = smem_base;                       // two Q tiles
+    const uint32_t sm_kv = smem_base + 2 * kTileBytes;     // kStages K/V tiles
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // ---- work item: (query tile, KV head of the group, pair of query heads) ---------------------
+    const int pairs = (p.G + 1) >> 1;
+    const int per_tile = p.Hg * pairs;
+    const int it = blockIdx.x / per_tile;
+    const int rem = blockIdx.x % per_tile;
+    const int hg = rem / pairs;
+    const int g0 = (rem % pairs) * 2;
+    const bool active1 = (g0 + 1) < p.G;
+    const int gt = p.total_tiles - 1 - it;      // long (late) tiles first
+    int b = 0;
+    while (b + 1 < p.B && gt >= p.tile_start[b + 1]) ++b;
+    const int qt = gt - p.tile_start[b];
+    const int r0 = qt * kTile;
+    const int C = p.n_new[b];
+    const int P = p.len[b];
+    const TilePlan plan = make_plan(p.kind, P, C, qt, p.S, p.W, p.ring);
+    const int n_tiles = plan.n_total;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&sh.q_full, 1);
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(&sh.kv_full[i], 1);
+            mbar_init(&sh.kv_empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&sh.s_full[i], 1);
+            mbar_init(&sh.p_full[i], 128);
+        }
+        mbar_init(&sh.o_full, 1);
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&sh.tmem_base))
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *(volatile uint32_t*)&sh.tmem_base;
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            const SeqDesc sd = p.desc[b];
+            const long long slots_per_head = (p.kind == ZZ_KIND_RETRIEVAL) ? sd.cap : p.ring;
+            const int k_row0 = (int)(sd.k_off[p.kind] / kD + (long long)hg * slots_per_head);
+            const int v_row0 = (int)(sd.v_off[p.kind] / kD + (long long)hg * slots_per_head);
+            const int src_head = p.head_list[p.kv_head0 + hg];
+            const int tok0 = p.tok_off[b];
+            const int qh = p.q_head0 + hg * p.G + g0;
+            mbar_expect_tx(&sh.q_full, active1 ? 2 * kTileBytes : kTileBytes);
+            tma_load_3d(sm_q, &tmap_q, 0, qh, tok0 + r0, &sh.q_full);
+            tma_load_3d(sm_q + kSubBytes, &tmap_q, 64, qh, tok0 + r0, &sh.q_full);
+            if (active1) {
+                tma_load_3d(sm_q + kTileBytes, &tmap_q, 0, qh + 1, tok0 + r0, &sh.q_full);
+                tma_load_3d(sm_q + kTileBytes + kSubBytes, &tmap_q, 64, qh + 1, tok0 + r0, &sh.q_full);
+            }
+            for (int u = 0; u < 2 * n_tiles; ++u) {
+                const int stage = u % kStages;
+                mbar_wait(&sh.kv_empty[stage], ((u / kStages) & 1) ^ 1, &sh, p.status);
+                bool is_chunk;
+                int start;
+                plan_tile(plan, u >> 1, is_chunk, start);
+                const bool is_v = u & 1;
+                const uint32_t dst = sm_kv + stage * kTileBytes;
+                mbar_expect_tx(&sh.kv_full[stage], kTileBytes);
+                if (is_chunk) {
+                    const CUtensorMap* m = is_v ? &tmap_v : &tmap_k;
+                    tma_load_3d(dst, m, 0, src_head, tok0 + start, &sh.kv_full[stage]);
+                    tma_load_3d(dst + kSubBytes, m, 64, src_head, tok0 + start, &sh.kv_full[stage]);
+                } else {
+                    const int row = (is_v ? v_row0 : k_row0) + start;
+                    tma_load_2d(dst, &tmap_arena, 0, row, &sh.kv_full[stage]);
+                    tma_load_2d(dst + kSubBytes, &tmap_arena, 64, row, &sh.kv_full[stage]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            const int n_act = active1 ? 2 : 1;
+            mbar_wait(&sh.q_full, 0, &sh, p.status);
+            mbar_wait(&sh.kv_full[0], 0, &sh, p.status);
+            tc_fence_after();
+            // S_t = Q_t K_0^T
+            for (int t = 0; t < n_act; ++t) {
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t off = (kk >> 2) * kSubBytes + (kk & 3) * 32;
+                    mma_ss(tmem + t * 256, make_desc(sm_q + t * kTileBytes + off, 16, 1024),
+                           make_desc(sm_kv + off, 16, 1024), kIdescQK, kk > 0);
+                }
+                mma_commit(&sh.s_full[t]);
+            }
+            mma_commit(&sh.kv_empty[0]);
+            for (int j = 0; j < n_tiles; ++j) {
+                const int uv = 2 * j + 1, uk = 2 * j + 2;
+                const int sv = uv % kStages, sk = uk % kStages;
+                const bool more = (j + 1) < n_tiles;
+                mbar_wait(&sh.kv_full[sv], (uv / kStages) & 1, &sh, p.status);
+                if (more) mbar_wait(&sh.kv_full[sk], (uk / kStages) & 1, &sh, p.status);
+                for (int t = 0; t < n_act; ++t) {
+                    mbar_wait(&sh.p_full[t], j & 1, &sh, p.status);
+                    tc_fence_after();
+                    // O_t (+)= P_t V_j
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        mma_ts(tmem + t * 256 + 128, tmem + t * 256 + kk * 8,
+                               make_desc(sm_kv + sv * kTileBytes + kk * 2048, kSubBytes, 1024), kIdescPV,
+                               (j > 0) || (kk > 0));
+                    }
+                    if (t == n_act - 1) mma_commit(&sh.kv_empty[sv]);
+                    if (more) {
+                        // S_t = Q_t K_{j+1}^T
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t off = (kk >> 2) * kSubBytes + (kk & 3) * 32;
+                            mma_ss(tmem + t * 256, make_desc(sm_q + t * kTileBytes + off, 16, 1024),
+                                   make_desc(sm_kv + sk * kTileBytes + off, 16, 1024), kIdescQK, kk > 0);
+                        }
+                        mma_commit(&sh.s_full[t]);
+                        if (t == n_act - 1) mma_commit(&sh.kv_empty[sk]);
+                    }
+                }
+            }
+            mma_commit(&sh.o_full);
+        }
+    } else {
+        // ================= softmax / correction / epilogue =================
+        const int t = (warp - 2) >> 2;                  // which of the two tiles
+        if (t == 0 || active1) {
+            const int quarter = warp & 3;               // tensor-memory lanes this warp may touch
+            const int r = quarter * 32 + lane;          // query row inside the tile
+            const int rr = r0 + r;                      // row inside the chunk
+            const uint32_t t_s = tmem + ((uint32_t)(quarter * 32) << 16) + t * 256;
+            const uint32_t t_o = t_s + 128;
+            const int* pos = p.pos + (long long)b * p.ring;
+            float m_used = -INFINITY, l_run = 0.f;
+            const float sc = p.scale_log2;
+            for (int j = 0; j < n_tiles; ++j) {
+                bool is_chunk;
+                int start;
+                plan_tile(plan, j, is_chunk, start);
+                mbar_wait(&sh.s_full[t], j & 1, &sh, p.status);
+                tc_fence_after();
+                float s[128];
+                tmem_ld32(t_s + 0, s + 0);
+                tmem_ld32(t_s + 32, s + 32);
+                tmem_ld32(t_s + 64, s + 64);
+                tmem_ld32(t_s + 96, s + 96);
+                tmem_wait_ld();
+
+                // ---- visibility ----------------------------------------------------------------
+                if (p.kind == ZZ_KIND_RETRIEVAL) {
+                    int lim = 128;                                    // columns [0, lim) are visible
+                    if (!is_chunk) lim = plan.n_occ - start;          // rows past the store's length
+                    else lim = rr - start + 1;                        // causal inside the chunk
+                    if (lim < 128) {
+#pragma unroll
+                        for (int c = 0; c < 128; ++c)
+                            if (c >= lim) s[c] = -INFINITY;
+                    }
+                } else if (!is_chunk) {
+                    const int tq = P + rr;
+#pragma unroll
+                    for (int c = 0; c < 128; ++c) {
+                        const int idx = start + c;
+                        bool ok = idx < plan.n_occ;
+                        if (ok) {
+                            const int pp = pos[idx];
+                            ok = (pp < p.S) || (tq - pp < p.W);
+                        }
+                        if (!ok) s[c] = -INFINITY;
+                    }
+                } else {
+                    const int c_hi = rr - start;                      // causal
+                    const int c_lo = rr - p.W + 1 - start;            // window
+                    const int c_sink = p.S - P - start;               // chunk tokens that are sinks
+#pragma unroll
+                    for (int c = 0; c < 128; ++c) {
+                        const bool ok = (c <= c_hi) && ((c >= c_lo) || (c < c_sink));
+                        if (!ok) s[c] = -INFINITY;
+                    }
+                }
+
+                // ---- running maximum, lazily applied ---------------------------------------------
+                float mx = s[0];
+#pragma unroll
+                for (int c = 1; c < 128; ++c) mx = fmaxf(mx, s[c]);
+                mx *= sc;
+                float alpha = 1.f;
+                bool bump = false;
+                if (mx > m_used + kRescaleThreshold || (m_used == -INFINITY && mx > -INFINITY)) {
+                    alpha = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - mx);
+                    m_used = mx;
+                    l_run *= alpha;
+                    bump = true;
+                }
+                if (j > 0 && __any_sync(0xffffffffu, bump)) {
+                    // PV of the previous tile has completed (its commit precedes s_full), so O is stable
+                    float o[32];
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        tmem_ld32(t_o + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] *= alpha;
+                        tmem_st32(t_o + c * 32, o);
+                    }
+                }
+                const float msub = (m_used == -INFINITY) ? 0.f : m_used;
+                float psum = 0.f;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float p0 = fast_exp2(fmaf(s[c * 32 + 2 * i], sc, -msub));
+                        const float p1 = fast_exp2(fmaf(s[c * 32 + 2 * i + 1], sc, -msub));
+                        psum += p0 + p1;
+                        pk[i] = pack_bf16(p0, p1);
+                    }
+                    tmem_st16(t_s + c * 16, pk);
+                }
+                l_run += psum;
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(&sh.p_full[t]);
+            }
+
+            // ---- epilogue: O / l -> bf16 -> global ---------------------------------------------------
+            mbar_wait(&sh.o_full, 0, &sh, p.status);
+            tc_fence_after();
+            const float inv = 1.f / l_run;
+            const bool row_ok = rr < C;
+            __nv_bfloat16* orow = p.out + (long long)(p.tok_off[b] + rr) * p.tok_stride +
+                                  (long long)(p.q_head0 + hg * p.G + g0 + t) * kD;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                float o[32];
+                tmem_ld32(t_o + c * 32, o);
+                tmem_wait_ld();
+                if (row_ok) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint4 w;
+                        w.x = pack_bf16(o[8 * i + 0] * inv, o[8 * i + 1] * inv);
+                        w.y = pack_bf16(o[8 * i + 2] * inv, o[8 * i + 3] * inv);
+                        w.z = pack_bf16(o[8 * i + 4] * inv, o[8 * i + 5] * inv);
+                        w.w = pack_bf16(o[8 * i + 6] * inv, o[8 * i + 7] * inv);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + i * 8) = w;
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        // every TMA load this CTA issued has been consumed (the MMA warp waited on each full
+        // barrier), and every MMA has completed (o_full); tensor memory can go back
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+    }
+}
+
+}  // namespace
+
+cudaError_t prefill_setup() {
+    return cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+}
+
+cudaError_t launch_prefill(const PrefillParams& p, const void* tq, const void* tk, const void* tv,
+                           const void* ta, int n_items, cudaStream_t s) {
+    prefill_kernel<<<n_items, kThreads, kSmemBytes, s>>>(p, *static_cast<const CUtensorMap*>(tq),
+                                                        *static_cast<const CUtensorMap*>(tk),
+                                                        *static_cast<const CUtensorMap*>(tv),
+                                                        *static_cast<const CUtensorMap*>(ta));
+    count_launch();
+    return cudaGetLastError();
+}
+
 }  // namespace zz
