@@ -137,6 +137,12 @@ int zz_decode_attn(zz_cache_t* cache, int layer, const void* d_q, void* d_out, v
 int zz_decode_step(zz_cache_t* cache, int layer, const void* d_q, const void* d_k,
                    const void* d_v, void* d_out, void* stream);
 
+/* One decode step of the whole stack: zz_decode_step for layers 0 .. n_layers-1 in order.
+ * d_q/d_out: [n_layers, batch, n_q_heads, 128]; d_k/d_v: [n_layers, batch, n_kv_heads, 128].
+ * Capacity is validated for every layer before anything is launched. */
+int zz_decode_step_all(zz_cache_t* cache, const void* d_q, const void* d_k, const void* d_v,
+                       void* d_out, void* stream);
+
 /* The same two calls fed from HOST memory: copies q/k/v into caller-provided device
  * staging (d_stage, at least zz_stage_bytes(cache, n_tokens) bytes), runs the call and
  * copies the result back to h_out.  Pinned host memory makes the copies asynchronous.
@@ -166,6 +172,16 @@ int zz_cache_import(zz_cache_t* cache, int layer, int seq, int kind, const void*
 /* Reads (and clears) the device status word: ZZ_OK, or ZZ_ERR_TIMEOUT if a bounded wait
  * inside a kernel expired since the last read.  Synchronises the stream. */
 int zz_get_last_status(zz_cache_t* cache, void* stream);
+
+/* Tracer (the paper has no counterpart; it reports per-token latencies only, Section 3.2).
+ * zz_profile_enable(n): n = 0 switches it off; n >= 1 brackets every n-th launch of each
+ * kernel class with two CUDA events on its stream (sampling keeps the host overhead low).
+ * zz_profile_read waits for the recorded events of one kernel class, returns how many
+ * launches were recorded and their summed device time, and (reset != 0) forgets all records.
+ * Classes: 0 append, 1 decode retrieval, 2 decode streaming, 3 prefill retrieval,
+ * 4 prefill streaming, 5 head regroup.  Process-wide, not thread-safe. */
+int zz_profile_enable(int period);
+int zz_profile_read(int kind, int64_t* launches, double* total_ms, int reset);
 
 /* Number of kernels this library has launched since it was loaded (all handles). */
 int64_t zz_launch_count(void);

@@ -70,6 +70,9 @@ SYMBOLS = {
     "zz_prefill_attn": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "zz_decode_attn": (_i32, [_vp, _i32, _vp, _vp, _vp]),
     "zz_decode_step": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp]),
+    "zz_decode_step_all": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "zz_profile_enable": (_i32, [_i32]),
+    "zz_profile_read": (_i32, [_i32, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double), _i32]),
     "zz_stage_bytes": (_sz, [_vp, _i64]),
     "zz_decode_step_host": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "zz_prefill_host": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
@@ -108,6 +111,30 @@ def version() -> int:
 
 def launch_count() -> int:
     return int(load().zz_launch_count())
+
+
+PROF_KINDS = {"append": 0, "decode_retrieval": 1, "decode_streaming": 2, "prefill_retrieval": 3,
+              "prefill_streaming": 4, "regroup": 5}
+
+
+def profile_enable(period: int) -> None:
+    """0 = off; n >= 1 = bracket every n-th launch of each kernel class with CUDA events."""
+    load().zz_profile_enable(int(period))
+
+
+def profile_read(reset: bool = True) -> dict:
+    """{kernel class: (launches, total device ms)} recorded since the last reset."""
+    lib = load()
+    out = {}
+    names = list(PROF_KINDS.items())
+    for i, (name, kind) in enumerate(names):
+        n, ms = ctypes.c_int64(0), ctypes.c_double(0.0)
+        last = i == len(names) - 1
+        rc = lib.zz_profile_read(kind, ctypes.byref(n), ctypes.byref(ms), 1 if (reset and last) else 0)
+        if rc != ZZ_OK:
+            raise ZigzagError(rc, "zz_profile_read")
+        out[name] = (int(n.value), float(ms.value))
+    return out
 
 
 def _check(status: int, what: str) -> None:
@@ -222,6 +249,10 @@ class ZigzagCache:
     def decode_step(self, layer: int, q, k, v, out, stream=None) -> None:
         _check(self._lib.zz_decode_step(self._h, layer, _dptr(q), _dptr(k), _dptr(v), _dptr(out),
                                         _stream_ptr(stream)), "zz_decode_step")
+
+    def decode_step_all(self, q, k, v, out, stream=None) -> None:
+        _check(self._lib.zz_decode_step_all(self._h, _dptr(q), _dptr(k), _dptr(v), _dptr(out),
+                                            _stream_ptr(stream)), "zz_decode_step_all")
 
     def stage_bytes(self, n_tokens: int) -> int:
         return int(self._lib.zz_stage_bytes(self._h, int(n_tokens)))

@@ -14,6 +14,39 @@
 namespace zz {
 static std::atomic<long long> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+// ---- tracer ------------------------------------------------------------------------------
+namespace {
+struct ProfRecord { int kind; cudaEvent_t e0, e1; };
+struct Profiler {
+    int period = 0;                  // 0 = off, n = sample every n-th launch of a class
+    long long seen[kProfKinds] = {0};
+    std::vector<ProfRecord> recs;
+    std::vector<cudaEvent_t> pool;   // events ready for reuse
+    cudaEvent_t pending = nullptr;
+    cudaEvent_t take() {
+        if (!pool.empty()) { cudaEvent_t e = pool.back(); pool.pop_back(); return e; }
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+        return e;
+    }
+} g_prof;
+}  // namespace
+void prof_begin(int kind, cudaStream_t s) {
+    g_prof.pending = nullptr;
+    if (g_prof.period <= 0) return;
+    if ((g_prof.seen[kind]++ % g_prof.period) != 0) return;
+    g_prof.pending = g_prof.take();
+    if (g_prof.pending) cudaEventRecord(g_prof.pending, s);
+}
+void prof_end(int kind, cudaStream_t s) {
+    if (!g_prof.pending) return;
+    cudaEvent_t e1 = g_prof.take();
+    if (!e1) { g_prof.pool.push_back(g_prof.pending); g_prof.pending = nullptr; return; }
+    cudaEventRecord(e1, s);
+    g_prof.recs.push_back(ProfRecord{kind, g_prof.pending, e1});
+    g_prof.pending = nullptr;
+}
 }  // namespace zz
 
 using zz::kD;
@@ -244,7 +277,11 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
     }
     plan_splits(c, n, Hg, &p.chunk, p.split_start);
     const int items = p.split_start[c->B] * Hg;
-    return zz::launch_decode(p, items, st) == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
+    const int pk = (kind == ZZ_KIND_RETRIEVAL) ? zz::kProfDecodeR : zz::kProfDecodeS;
+    zz::prof_begin(pk, st);
+    const cudaError_t e = zz::launch_decode(p, items, st);
+    zz::prof_end(pk, st);
+    return e == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
 }
 
 int regroup(zz_cache* c, int layer, const __nv_bfloat16* src, __nv_bfloat16* dst, long long tokens,
@@ -257,7 +294,10 @@ int regroup(zz_cache* c, int layer, const __nv_bfloat16* src, __nv_bfloat16* dst
     g.G = c->G;
     g.tokens = tokens;
     g.to_compact = to_compact;
-    return zz::launch_regroup(g, st) == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
+    zz::prof_begin(zz::kProfRegroup, st);
+    const cudaError_t e = zz::launch_regroup(g, st);
+    zz::prof_end(zz::kProfRegroup, st);
+    return e == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
 }
 
 int launch_prefill_group(zz_cache* c, int layer, int kind, const CUtensorMap* tq, const CUtensorMap* tk,
@@ -300,8 +340,11 @@ int launch_prefill_group(zz_cache* c, int layer, int kind, const CUtensorMap* tq
     const long long items = (long long)tiles * Hg * pairs;
     if (items == 0) return ZZ_OK;
     if (items > 0x7fffffffLL) return ZZ_ERR_UNSUPPORTED;
-    return zz::launch_prefill(p, tq, tk, tv, &c->tmap_arena, (int)items, st) == cudaSuccess ? ZZ_OK
-                                                                                             : ZZ_ERR_CUDA;
+    const int pk = (kind == ZZ_KIND_RETRIEVAL) ? zz::kProfPrefillR : zz::kProfPrefillS;
+    zz::prof_begin(pk, st);
+    const cudaError_t e = zz::launch_prefill(p, tq, tk, tv, &c->tmap_arena, (int)items, st);
+    zz::prof_end(pk, st);
+    return e == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
 }
 
 }  // namespace
@@ -469,7 +512,10 @@ int zz_kv_append(zz_cache_t* c, int layer, const void* d_k, const void* d_v, con
     }
     const long long gx = (worst + 255) / 256;
     if (gx > 0x7fffffffLL) return ZZ_ERR_UNSUPPORTED;
-    if (zz::launch_append(p, (int)gx, static_cast<cudaStream_t>(stream)) != cudaSuccess) return ZZ_ERR_CUDA;
+    zz::prof_begin(zz::kProfAppend, static_cast<cudaStream_t>(stream));
+    const cudaError_t ae = zz::launch_append(p, (int)gx, static_cast<cudaStream_t>(stream));
+    zz::prof_end(zz::kProfAppend, static_cast<cudaStream_t>(stream));
+    if (ae != cudaSuccess) return ZZ_ERR_CUDA;
     for (int b = 0; b < c->B; ++b) c->len[(size_t)layer * c->B + b] += h_n_new[b];
     return ZZ_OK;
 }
@@ -504,6 +550,55 @@ int zz_decode_step(zz_cache_t* c, int layer, const void* d_q, const void* d_k, c
     const int r = zz_kv_append(c, layer, d_k, d_v, ones, stream);
     if (r != ZZ_OK) return r;
     return zz_decode_attn(c, layer, d_q, d_out, stream);
+}
+
+int zz_decode_step_all(zz_cache_t* c, const void* d_q, const void* d_k, const void* d_v, void* d_out,
+                       void* stream) {
+    if (!c || !d_q || !d_k || !d_v || !d_out) return ZZ_ERR_INVALID_ARG;
+    const size_t qs = (size_t)c->B * c->Hq * kD * 2, ks = (size_t)c->B * c->Hkv * kD * 2;
+    // validate every layer before launching anything
+    for (int l = 0; l < c->L; ++l)
+        for (int b = 0; b < c->B; ++b)
+            if (c->nR[l] > 0 && c->len[(size_t)l * c->B + b] + 1 > c->cap[b]) return ZZ_ERR_CAPACITY;
+    for (int l = 0; l < c->L; ++l) {
+        const int r = zz_decode_step(c, l, static_cast<const char*>(d_q) + l * qs,
+                                     static_cast<const char*>(d_k) + l * ks,
+                                     static_cast<const char*>(d_v) + l * ks,
+                                     static_cast<char*>(d_out) + l * qs, stream);
+        if (r != ZZ_OK) return r;
+    }
+    return ZZ_OK;
+}
+
+int zz_profile_enable(int period) {
+    if (period < 0) return ZZ_ERR_INVALID_ARG;
+    zz::g_prof.period = period;
+    for (int i = 0; i < zz::kProfKinds; ++i) zz::g_prof.seen[i] = 0;
+    return ZZ_OK;
+}
+
+int zz_profile_read(int kind, int64_t* launches, double* total_ms, int reset) {
+    if (kind < 0 || kind >= zz::kProfKinds || !launches || !total_ms) return ZZ_ERR_INVALID_ARG;
+    long long n = 0;
+    double ms = 0.0;
+    for (const auto& r : zz::g_prof.recs) {
+        if (r.kind != kind) continue;
+        if (cudaEventSynchronize(r.e1) != cudaSuccess) return ZZ_ERR_CUDA;
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, r.e0, r.e1) != cudaSuccess) return ZZ_ERR_CUDA;
+        ms += t;
+        ++n;
+    }
+    *launches = n;
+    *total_ms = ms;
+    if (reset) {
+        for (const auto& r : zz::g_prof.recs) {
+            zz::g_prof.pool.push_back(r.e0);
+            zz::g_prof.pool.push_back(r.e1);
+        }
+        zz::g_prof.recs.clear();
+    }
+    return ZZ_OK;
 }
 
 int zz_prefill_attn(zz_cache_t* c, int layer, const void* d_q, const void* d_k, const void* d_v, void* d_out,

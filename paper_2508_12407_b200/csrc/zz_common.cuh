@@ -103,4 +103,11 @@ cudaError_t launch_prefill(const PrefillParams& p, const void* tmap_q, const voi
 
 void count_launch(int n = 1);
 
+// Lightweight tracer: when enabled, every launch is bracketed by two CUDA events on its
+// stream and accumulated per kernel class.
+enum ProfKind { kProfAppend = 0, kProfDecodeR = 1, kProfDecodeS = 2, kProfPrefillR = 3, kProfPrefillS = 4,
+                kProfRegroup = 5, kProfOther = 6, kProfKinds = 7 };
+void prof_begin(int kind, cudaStream_t s);
+void prof_end(int kind, cudaStream_t s);
+
 }  // namespace zz
