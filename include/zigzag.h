@@ -104,8 +104,11 @@ int zz_cache_reset(zz_cache_t* cache, int seq, void* stream);
 /* Host-mirrored length of (layer, seq). */
 int zz_cache_len(const zz_cache_t* cache, int layer, int seq, int32_t* len);
 
-/* Tuning knob for experiments; the paper has no counterpart.  Keys: "decode_min_chunk"
- * (fewest tokens per split of the decode kernel; a multiple of 16, default 256). */
+/* Tuning knobs for experiments; the paper has no counterpart.  Keys: "decode_min_chunk"
+ * (fewest tokens per split of the long-store decode plan; a multiple of 16, default 256);
+ * "decode_short_tokens" (tokens per CTA of the short-store plan, and the threshold
+ * total_tokens * kv_heads <= SMs * value below which it is used; multiple of 16, default
+ * 384; 0 disables the short-store plan). */
 int zz_tune(zz_cache_t* cache, const char* key, int value);
 
 /* KV append with sink + recent eviction (paper: Introduction -- the KV cache grows with

@@ -54,7 +54,7 @@ using zz::SeqDesc;
 
 namespace {
 
-constexpr int kMaxSplits = 128;
+constexpr int kMaxSplits = 120;   // the decode kernel keeps per-split factors in 128-entry rows
 constexpr size_t kAlign = 256;
 
 size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
@@ -127,6 +127,7 @@ struct zz_cache {
     unsigned char* work;
     int num_sms;
     int decode_min_chunk;
+    int decode_short_tokens;
     bool has_mixed;
     alignas(64) CUtensorMap tmap_arena;
     bool have_tmap_arena;
@@ -206,7 +207,7 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
     lay->off_pos = w; w += align_up((size_t)L * B * ring * sizeof(int));
     lay->off_desc = w; w += align_up((size_t)L * B * sizeof(SeqDesc));
     lay->off_heads = w; w += align_up((size_t)L * Hkv * sizeof(int));
-    lay->off_counters = w; w += align_up((size_t)B * Hkv * sizeof(unsigned int));
+    lay->off_counters = w; w += align_up((size_t)(B * Hkv + B) * sizeof(unsigned int));
     lay->off_part_ml = w; w += align_up((size_t)B * Hkv * kMaxSplits * G * 2 * sizeof(float));
     lay->off_part_o = w; w += align_up((size_t)B * Hkv * kMaxSplits * G * kD * sizeof(float));
     lay->off_qc = w;
@@ -218,43 +219,68 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
 
 bool bad_layer(const zz_cache* c, int layer) { return !c || layer < 0 || layer >= c->L; }
 
-// Tokens per split and per-sequence split counts so that all work items fit one wave.
-void plan_splits(const zz_cache* c, const int* n, int Hg, int* chunk_out, int* split_start) {
-    const int slots = 2 * c->num_sms;
+// Split plan of one decode launch.  Short stores: 8-warp CTAs (one per SM) that each take up to
+// 384 tokens, so a warp's chain is at most three dependent steps.  Long stores: 4-warp CTAs
+// (two per SM), all work items in one wave, every sequence cut into equal splits.
+void plan_splits(const zz_cache* c, const int* n, int Hg, int* warps, int* chunk, int* split_start) {
     long long total = 0;
     for (int b = 0; b < c->B; ++b) total += n[b];
-    long long chunk = (total * Hg + slots - 1) / slots;
-    chunk = (chunk + 63) / 64 * 64;
-    if (chunk < c->decode_min_chunk) chunk = c->decode_min_chunk;
+    split_start[0] = 0;
+    if (total * Hg <= (long long)c->num_sms * c->decode_short_tokens) {
+        *warps = 8;
+        for (int b = 0; b < c->B; ++b) {
+            int s = (n[b] + c->decode_short_tokens - 1) / c->decode_short_tokens;
+            if (s < 1) s = 1;
+            chunk[b] = c->decode_short_tokens;
+            split_start[b + 1] = split_start[b] + s;
+        }
+        return;
+    }
+    *warps = 4;
+    const int slots = 2 * c->num_sms;
+    long long per = (total * Hg + slots - 1) / slots;   // tokens per work item if all were equal
+    if (per < c->decode_min_chunk) per = c->decode_min_chunk;
     for (;;) {
         long long items = 0;
         int worst = 0;
         for (int b = 0; b < c->B; ++b) {
-            const int s = (int)((n[b] + chunk - 1) / chunk);
+            const int s = (int)((n[b] + per - 1) / per);
             items += (long long)(s > 0 ? s : 1) * Hg;
             if (s > worst) worst = s;
         }
-        if ((items <= slots || chunk >= total) && worst <= kMaxSplits) break;
-        chunk += 64;
+        if ((items <= slots || per >= total) && worst <= kMaxSplits) break;
+        per += 16;
     }
-    split_start[0] = 0;
     for (int b = 0; b < c->B; ++b) {
-        int s = (int)((n[b] + chunk - 1) / chunk);
+        int s = (int)((n[b] + per - 1) / per);
         if (s < 1) s = 1;
+        chunk[b] = (n[b] + s - 1) / s;            // equal splits inside the sequence
+        if (chunk[b] < 1) chunk[b] = 1;
         split_start[b + 1] = split_start[b] + s;
     }
-    *chunk_out = (int)chunk;
 }
 
+// k_new/v_new != nullptr: fused append of one token per sequence (host lengths not yet bumped)
 int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q, __nv_bfloat16* out,
-                        int q_head0, cudaStream_t st) {
+                        int q_head0, cudaStream_t st, const __nv_bfloat16* k_new = nullptr,
+                        const __nv_bfloat16* v_new = nullptr, int bump_len = 0) {
     const int Hg = (kind == ZZ_KIND_RETRIEVAL) ? c->nR[layer] : c->Hkv - c->nR[layer];
     if (Hg == 0) return ZZ_OK;
     zz::DecodeParams p;
     memset(&p, 0, sizeof p);
     p.arena = c->d_arena();
-    p.desc = c->d_desc(layer);
     p.len = c->d_len(layer);
+    for (int b = 0; b < c->B; ++b) p.sd[b] = c->desc[(size_t)layer * c->B + b];
+    p.k_new = k_new;
+    p.v_new = v_new;
+    p.head_list = c->d_heads(layer);
+    p.pos = c->d_pos(layer);
+    p.seq_counters = c->d_counters() + (size_t)c->B * c->Hkv;
+    p.kv_head0 = (kind == ZZ_KIND_RETRIEVAL) ? 0 : c->nR[layer];
+    p.n_kv_total = c->Hkv;
+    p.S = c->S;
+    p.W = c->W;
+    p.bump_len = bump_len;
     p.q = q;
     p.out = out;
     p.q_tok_stride = (long long)c->Hq * kD;
@@ -272,14 +298,15 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
     p.scale_log2 = c->scale * 1.4426950408889634f;
     int n[ZZ_MAX_BATCH];
     for (int b = 0; b < c->B; ++b) {
-        const int len = c->len[(size_t)layer * c->B + b];
+        const int len = c->len[(size_t)layer * c->B + b] + (k_new ? 1 : 0);
         n[b] = (kind == ZZ_KIND_RETRIEVAL) ? len : (len < c->ring ? len : c->ring);
     }
-    plan_splits(c, n, Hg, &p.chunk, p.split_start);
+    int warps = 4;
+    plan_splits(c, n, Hg, &warps, p.chunk, p.split_start);
     const int items = p.split_start[c->B] * Hg;
     const int pk = (kind == ZZ_KIND_RETRIEVAL) ? zz::kProfDecodeR : zz::kProfDecodeS;
     zz::prof_begin(pk, st);
-    const cudaError_t e = zz::launch_decode(p, items, st);
+    const cudaError_t e = zz::launch_decode(p, items, warps, st);
     zz::prof_end(pk, st);
     return e == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
 }
@@ -391,6 +418,7 @@ int zz_cache_create(const zz_config_t* cfg, void* d_arena, size_t arena_bytes, v
     c->G = c->Hq / c->Hkv; c->S = cfg->sink; c->W = cfg->recent; c->ring = c->S + c->W;
     c->max_new = cfg->max_new_tokens; c->scale = cfg->softmax_scale;
     c->decode_min_chunk = 256;
+    c->decode_short_tokens = 384;
     compute_layout(cfg, &c->lay, &c->desc);
     if (arena_bytes < c->lay.arena_bytes || workspace_bytes < c->lay.work_bytes) {
         delete c;
@@ -473,6 +501,11 @@ int zz_tune(zz_cache_t* c, const char* key, int value) {
         c->decode_min_chunk = value;
         return ZZ_OK;
     }
+    if (!strcmp(key, "decode_short_tokens")) {
+        if (value < 0 || value % 16) return ZZ_ERR_INVALID_ARG;
+        c->decode_short_tokens = value;
+        return ZZ_OK;
+    }
     return ZZ_ERR_INVALID_ARG;
 }
 
@@ -543,13 +576,34 @@ int zz_decode_attn(zz_cache_t* c, int layer, const void* d_q, void* d_out, void*
 
 int zz_decode_step(zz_cache_t* c, int layer, const void* d_q, const void* d_k, const void* d_v, void* d_out,
                    void* stream) {
-    if (bad_layer(c, layer)) return ZZ_ERR_INVALID_ARG;
-    int32_t ones[ZZ_MAX_BATCH];
-    for (int b = 0; b < c->B; ++b) ones[b] = 1;
-    if (!d_q || !d_out) return ZZ_ERR_INVALID_ARG;
-    const int r = zz_kv_append(c, layer, d_k, d_v, ones, stream);
+    if (bad_layer(c, layer) || !d_q || !d_k || !d_v || !d_out) return ZZ_ERR_INVALID_ARG;
+    if (((uintptr_t)d_q | (uintptr_t)d_k | (uintptr_t)d_v | (uintptr_t)d_out) & 15) return ZZ_ERR_INVALID_ARG;
+    const int nR = c->nR[layer];
+    for (int b = 0; b < c->B; ++b) {
+        const long long nl = (long long)c->len[(size_t)layer * c->B + b] + 1;
+        if (nl > 0x7fffffffLL || (nR > 0 && nl > c->cap[b])) return ZZ_ERR_CAPACITY;
+    }
+    // the append is fused into the attention kernel: the new row is read from d_k/d_v, stored in
+    // its slot and attended to by the same launch
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(d_q);
+    const __nv_bfloat16* k = static_cast<const __nv_bfloat16*>(d_k);
+    const __nv_bfloat16* v = static_cast<const __nv_bfloat16*>(d_v);
+    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(d_out);
+    int r;
+    if (!c->mixed(layer)) {
+        const int kind = nR ? ZZ_KIND_RETRIEVAL : ZZ_KIND_STREAMING;
+        r = launch_decode_group(c, layer, kind, q, out, 0, st, k, v, 1);
+    } else {
+        r = regroup(c, layer, q, c->d_qc(), c->B, 1, st);
+        if (r == ZZ_OK) r = launch_decode_group(c, layer, ZZ_KIND_RETRIEVAL, c->d_qc(), c->d_oc(), 0, st, k, v, 0);
+        if (r == ZZ_OK)
+            r = launch_decode_group(c, layer, ZZ_KIND_STREAMING, c->d_qc(), c->d_oc(), nR * c->G, st, k, v, 1);
+        if (r == ZZ_OK) r = regroup(c, layer, c->d_oc(), out, c->B, 0, st);
+    }
     if (r != ZZ_OK) return r;
-    return zz_decode_attn(c, layer, d_q, d_out, stream);
+    for (int b = 0; b < c->B; ++b) c->len[(size_t)layer * c->B + b] += 1;
+    return ZZ_OK;
 }
 
 int zz_decode_step_all(zz_cache_t* c, const void* d_q, const void* d_k, const void* d_v, void* d_out,

@@ -38,9 +38,8 @@ struct AppendParams {
 };
 
 struct DecodeParams {
-    const __nv_bfloat16* arena;
-    const SeqDesc* desc;     // [B]
-    const int* len;          // [B]
+    __nv_bfloat16* arena;
+    int* len;                // [B] device lengths of this layer
     const __nv_bfloat16* q;  // row of sequence b, head h at q + b*q_tok_stride + (q_head0 + h)*128
     __nv_bfloat16* out;      // same addressing as q
     long long q_tok_stride;  // elements between consecutive sequences' rows (n_q_heads * 128)
@@ -52,10 +51,22 @@ struct DecodeParams {
     int kind;                // which group of the layer
     int ring;                // S+W
     int Hg, G, B;
-    int chunk;               // tokens per split (multiple of 16)
     int max_splits;
     float scale_log2;        // softmax_scale * log2(e)
+    // fused append (k_new != nullptr): the token at position len is taken from k_new/v_new
+    // ([B][n_kv_total][128], model head order), written to its slot, and attended to
+    const __nv_bfloat16* k_new;
+    const __nv_bfloat16* v_new;
+    const int* head_list;    // [n_kv_total] group-ordered source KV heads
+    int* pos;                // [B][ring] ring positions of this layer
+    unsigned int* seq_counters;  // [B], 0 between launches
+    int kv_head0;            // first entry of head_list that belongs to the group
+    int n_kv_total;
+    int S, W;
+    int bump_len;            // this launch advances len (the last launch of a layer does)
     int split_start[ZZ_MAX_BATCH + 1];  // prefix sum of per-sequence split counts
+    int chunk[ZZ_MAX_BATCH];            // tokens per split of each sequence
+    SeqDesc sd[ZZ_MAX_BATCH];           // store addresses of every sequence of this layer
 };
 
 struct GatherParams {
@@ -91,7 +102,7 @@ struct PrefillParams {
 
 // ---- launchers (defined in the .cu files) -------------------------------------------
 cudaError_t launch_append(const AppendParams& p, int grid_x, cudaStream_t s);
-cudaError_t launch_decode(const DecodeParams& p, int n_items, cudaStream_t s);
+cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStream_t s);
 cudaError_t launch_regroup(const GatherParams& p, cudaStream_t s);
 cudaError_t launch_reset(int* len, int* pos, int L, int B, int ring, int seq, cudaStream_t s);
 cudaError_t decode_setup();

@@ -20,12 +20,12 @@ namespace zz {
 
 namespace {
 
-constexpr int kWarps = 4;
 constexpr int kBlk = 16;                       // tokens per warp step
 constexpr int kStages = 3;
 constexpr int kStageBytes = kBlk * kRowBytes;  // 4 KiB of K (and as much of V) per stage
-constexpr int kWarpSmem = kStages * 2 * kStageBytes;
-constexpr int kSmemBytes = kWarps * kWarpSmem;  // 96 KiB -> two CTAs per SM
+constexpr int kWarpSmem = kStages * 2 * kStageBytes;   // 24 KiB per warp
+// 4 warps: 96 KiB, two CTAs per SM (long contexts); 8 warps: 192 KiB, one CTA per SM (short
+// stores, where the per-warp chain of dependent steps is what costs)
 constexpr int kMaxSplitsSmem = 128;             // >= the host's split limit
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -78,8 +78,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 // Issue the loads of one 16-token block (K and V rows of one head) into a stage.
 // Row r, 16-byte piece c lands at r*256 + ((c ^ (r & 7)) * 16): conflict-free for ldmatrix.
+// Slot `new_slot` (if inside the block) is the token being appended by this very launch: its
+// row comes from the caller's k_new/v_new instead of the store.
 __device__ __forceinline__ void load_block(uint32_t stage_k, uint32_t stage_v, const __nv_bfloat16* kbase,
-                                           const __nv_bfloat16* vbase, int tok0, int tok_end, int lane) {
+                                           const __nv_bfloat16* vbase, int tok0, int tok_end, int lane,
+                                           int new_slot, const __nv_bfloat16* knew, const __nv_bfloat16* vnew) {
 #pragma unroll
     for (int it = 0; it < 8; ++it) {
         const int idx = it * 32 + lane;
@@ -88,14 +91,15 @@ __device__ __forceinline__ void load_block(uint32_t stage_k, uint32_t stage_v, c
         const int ok = tok < tok_end;
         const long long off = (long long)(ok ? tok : tok0) * kD + c * 8;
         const uint32_t so = r * kRowBytes + ((c ^ (r & 7)) << 4);
-        cp_async16(stage_k + so, kbase + off, ok ? 16 : 0);
-        cp_async16(stage_v + so, vbase + off, ok ? 16 : 0);
+        const bool fresh = tok == new_slot;
+        cp_async16(stage_k + so, fresh ? knew + c * 8 : kbase + off, ok ? 16 : 0);
+        cp_async16(stage_v + so, fresh ? vnew + c * 8 : vbase + off, ok ? 16 : 0);
     }
 }
 
 // HI = group size above 8 (rows 8..15 of the tile carry query heads too).
-template <bool HI>
-__global__ void __launch_bounds__(kWarps * 32, 2) decode_kernel(const DecodeParams p) {
+template <bool HI, int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const DecodeParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     __shared__ int s_is_last;
 
@@ -111,17 +115,37 @@ __global__ void __launch_bounds__(kWarps * 32, 2) decode_kernel(const DecodePara
     const int split = local / p.Hg;
     const int nsplit = p.split_start[b + 1] - p.split_start[b];
 
-    const SeqDesc sd = p.desc[b];
-    const int len = p.len[b];
+    const bool fused = p.k_new != nullptr;
+    const int len_old = p.len[b];
+    const int len = len_old + (fused ? 1 : 0);
     const int n = (p.kind == ZZ_KIND_RETRIEVAL) ? len : min(len, p.ring);
-    const long long slots_per_head = (p.kind == ZZ_KIND_RETRIEVAL) ? sd.cap : p.ring;
-    const __nv_bfloat16* kbase = p.arena + sd.k_off[p.kind] + (long long)hg * slots_per_head * kD;
-    const __nv_bfloat16* vbase = p.arena + sd.v_off[p.kind] + (long long)hg * slots_per_head * kD;
+    const long long slots_per_head = (p.kind == ZZ_KIND_RETRIEVAL) ? p.sd[b].cap : p.ring;
+    __nv_bfloat16* kbase = p.arena + p.sd[b].k_off[p.kind] + (long long)hg * slots_per_head * kD;
+    __nv_bfloat16* vbase = p.arena + p.sd[b].v_off[p.kind] + (long long)hg * slots_per_head * kD;
+    int new_slot = -1;
+    const __nv_bfloat16* knew = nullptr;
+    const __nv_bfloat16* vnew = nullptr;
+    if (fused) {
+        const int t = len_old;
+        new_slot = (p.kind == ZZ_KIND_RETRIEVAL || t < p.S) ? t : p.S + ((t - p.S) % p.W);
+        const long long src = ((long long)b * p.n_kv_total + p.head_list[p.kv_head0 + hg]) * kD;
+        knew = p.k_new + src;
+        vnew = p.v_new + src;
+    }
 
-    const int s0 = min(split * p.chunk, n);
-    const int s1 = (split == nsplit - 1) ? n : min(n, s0 + p.chunk);
+    const int s0 = min(split * p.chunk[b], n);
+    const int s1 = (split == nsplit - 1) ? n : min(n, s0 + p.chunk[b]);
     const int nblk = (s1 - s0 + kBlk - 1) / kBlk;              // 16-token blocks of this CTA
     const int my_blocks = (nblk > warp) ? (nblk - warp + kWarps - 1) / kWarps : 0;
+
+    // ---- fused append: the CTA whose range holds the new slot stores the row ----------------
+    if (fused && new_slot >= s0 && new_slot < s1 && warp == kWarps - 1) {
+        const int c = lane & 15;
+        const __nv_bfloat16* src = (lane < 16 ? knew : vnew) + c * 8;
+        __nv_bfloat16* dst = (lane < 16 ? kbase : vbase) + (long long)new_slot * kD + c * 8;
+        *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+        if (p.kind == ZZ_KIND_STREAMING && hg == 0 && lane == 0) p.pos[(long long)b * p.ring + new_slot] = len_old;
+    }
 
     // ---- query fragments: rows = the G heads of this KV head ---------------------------
     const int G = p.G;
@@ -157,7 +181,7 @@ __global__ void __launch_bounds__(kWarps * 32, 2) decode_kernel(const DecodePara
         if (s < my_blocks) {
             const int tok0 = s0 + (warp + s * kWarps) * kBlk;
             load_block(wbase + s * 2 * kStageBytes, wbase + s * 2 * kStageBytes + kStageBytes, kbase, vbase,
-                       tok0, s1, lane);
+                       tok0, s1, lane, new_slot, knew, vnew);
         }
         cp_async_commit();
     }
@@ -169,7 +193,7 @@ __global__ void __launch_bounds__(kWarps * 32, 2) decode_kernel(const DecodePara
                 const int st = nx % kStages;
                 const int tok0 = s0 + (warp + nx * kWarps) * kBlk;
                 load_block(wbase + st * 2 * kStageBytes, wbase + st * 2 * kStageBytes + kStageBytes, kbase,
-                           vbase, tok0, s1, lane);
+                           vbase, tok0, s1, lane, new_slot, knew, vnew);
             }
             cp_async_commit();
         }
@@ -273,10 +297,10 @@ __global__ void __launch_bounds__(kWarps * 32, 2) decode_kernel(const DecodePara
     }
     __syncthreads();
 
-    const int d = threadIdx.x;   // 128 threads = 128 output dims
+    const int d = threadIdx.x & 127;   // 128 output dims; with 8 warps the halves split the rows
     const long long pair = (long long)b * p.Hg + hg;
     __nv_bfloat16* outb = p.out + ((long long)b * p.q_tok_stride) + (long long)(p.q_head0 + hg * G) * kD;
-    for (int row = 0; row < G; ++row) {
+    for (int row = threadIdx.x >> 7; row < G; row += kWarps / 4) {
         float M = -INFINITY;
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) M = fmaxf(M, sm_ml[(w * 16 + row) * 2]);
@@ -299,6 +323,19 @@ __global__ void __launch_bounds__(kWarps * 32, 2) decode_kernel(const DecodePara
             }
         }
     }
+    if (fused && p.bump_len) {
+        // every CTA of the sequence has read the old length by the time it gets here; the last
+        // one to arrive publishes the new length
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const unsigned int all = (unsigned int)(nsplit * p.Hg);
+            const unsigned int prev = atomicAdd(p.seq_counters + b, 1u);
+            if (prev == all - 1) {
+                p.len[b] = len_old + 1;
+                p.seq_counters[b] = 0u;
+            }
+        }
+    }
     if (nsplit == 1) return;
 
     // ---- last CTA of this (sequence, head) merges the splits -----------------------------------
@@ -311,43 +348,69 @@ __global__ void __launch_bounds__(kWarps * 32, 2) decode_kernel(const DecodePara
     __syncthreads();
     if (!s_is_last) return;
     __threadfence();
-    // (max, sum) of every split and row into shared memory, then each thread owns one output
-    // dimension and streams the partial outputs with independent loads in flight
-    float* sm_m = reinterpret_cast<float*>(smem);            // [G][nsplit]
-    float* sm_f = sm_m + 16 * kMaxSplitsSmem;                // [G][nsplit] -> scale factors
-    for (int i = threadIdx.x; i < nsplit * G; i += blockDim.x) {
-        const int s = i / G, row = i % G;
-        const long long po = ((pair * p.max_splits + s) * G + row);
-        sm_m[row * kMaxSplitsSmem + s] = __ldcg(p.part_ml + po * 2);
-        sm_f[row * kMaxSplitsSmem + s] = __ldcg(p.part_ml + po * 2 + 1);
-    }
-    __syncthreads();
-    for (int row = 0; row < G; ++row) {
-        float M = -INFINITY;
-        for (int s = 0; s < nsplit; ++s) M = fmaxf(M, sm_m[row * kMaxSplitsSmem + s]);
-        float L = 0.f, acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
-        const float* po = p.part_o + ((pair * p.max_splits) * G + row) * kD + d;
+    // Merge of the splits in (about) one memory round trip: thread (row, 4 dims) first issues the
+    // float4 loads of every split's partial output, then the (max, sum) pairs are turned into
+    // per-split factors through shared memory while those loads are in flight.
+    float* sm_m = reinterpret_cast<float*>(smem);            // [16][128] running max per split
+    float* sm_f = sm_m + 16 * kMaxSplitsSmem;                // [16][128] sum, then factor
+    constexpr int kRound = 32;                               // splits whose partials are held at once
+    for (int row0 = 0; row0 < G; row0 += kWarps) {
+        const int row = row0 + warp;                         // this warp's row (4 dims per lane)
+        const bool row_ok = row < G;
+        const float* pbase = p.part_o + ((pair * p.max_splits) * G + (row_ok ? row : 0)) * kD + lane * 4;
         const long long sstride = (long long)G * kD;
-        int s = 0;
-        for (; s + 4 <= nsplit; s += 4) {
-            const float v0 = __ldcg(po + (s + 0) * sstride), v1 = __ldcg(po + (s + 1) * sstride);
-            const float v2 = __ldcg(po + (s + 2) * sstride), v3 = __ldcg(po + (s + 3) * sstride);
-            float f[4];
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int sb = 0; sb < nsplit; sb += kRound) {
+            float4 v[kRound];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const float ms = sm_m[row * kMaxSplitsSmem + s + u];
-                f[u] = (ms == -INFINITY) ? 0.f : fast_exp2(ms - M);
-                L += f[u] * sm_f[row * kMaxSplitsSmem + s + u];
+            for (int u = 0; u < kRound; ++u)
+                v[u] = (row_ok && sb + u < nsplit) ? __ldcg(reinterpret_cast<const float4*>(pbase + (sb + u) * sstride))
+                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+            if (sb == 0) {
+                for (int i = threadIdx.x; i < nsplit * kWarps; i += blockDim.x) {
+                    const int s = i / kWarps, r = row0 + i % kWarps;
+                    if (r < G) {
+                        const long long po = ((pair * p.max_splits + s) * G + r);
+                        const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + po * 2));
+                        sm_m[r * kMaxSplitsSmem + s] = ml.x;
+                        sm_f[r * kMaxSplitsSmem + s] = ml.y;
+                    }
+                }
+                __syncthreads();
+                if (row_ok) {
+                    float M = -INFINITY;
+                    for (int s = lane; s < nsplit; s += 32) M = fmaxf(M, sm_m[row * kMaxSplitsSmem + s]);
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+                    float L = 0.f;
+                    for (int s = lane; s < nsplit; s += 32) {
+                        const float ms = sm_m[row * kMaxSplitsSmem + s];
+                        const float f = (ms == -INFINITY) ? 0.f : fast_exp2(ms - M);
+                        L += f * sm_f[row * kMaxSplitsSmem + s];
+                        sm_f[row * kMaxSplitsSmem + s] = f;
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+                    if (lane == 0) sm_m[row * kMaxSplitsSmem + kMaxSplitsSmem - 1] = 1.f / L;  // slot no split uses
+                }
+                __syncwarp();
             }
-            acc0 += f[0] * v0; acc1 += f[1] * v1; acc2 += f[2] * v2; acc3 += f[3] * v3;
+#pragma unroll
+            for (int u = 0; u < kRound; ++u) {
+                if (row_ok && sb + u < nsplit) {
+                    const float f = sm_f[row * kMaxSplitsSmem + sb + u];
+                    acc.x += f * v[u].x; acc.y += f * v[u].y; acc.z += f * v[u].z; acc.w += f * v[u].w;
+                }
+            }
         }
-        for (; s < nsplit; ++s) {
-            const float ms = sm_m[row * kMaxSplitsSmem + s];
-            const float f = (ms == -INFINITY) ? 0.f : fast_exp2(ms - M);
-            L += f * sm_f[row * kMaxSplitsSmem + s];
-            acc0 += f * __ldcg(po + s * sstride);
+        if (row_ok) {
+            const float inv = sm_m[row * kMaxSplitsSmem + kMaxSplitsSmem - 1];
+            uint2 w;
+            w.x = pack_bf16(acc.x * inv, acc.y * inv);
+            w.y = pack_bf16(acc.z * inv, acc.w * inv);
+            *reinterpret_cast<uint2*>(outb + row * kD + lane * 4) = w;
         }
-        outb[row * kD + d] = __float2bfloat16_rn(((acc0 + acc1) + (acc2 + acc3)) / L);
+        __syncthreads();
     }
     if (threadIdx.x == 0) p.counters[pair] = 0u;
 }
@@ -355,18 +418,30 @@ __global__ void __launch_bounds__(kWarps * 32, 2) decode_kernel(const DecodePara
 }  // namespace
 
 cudaError_t decode_setup() {
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kSmemBytes);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(decode_kernel<false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         4 * kWarpSmem);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(decode_kernel<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * kWarpSmem);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(decode_kernel<false, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * kWarpSmem);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(decode_kernel<true, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * kWarpSmem);
+    return e;
 }
 
-cudaError_t launch_decode(const DecodeParams& p, int n_items, cudaStream_t s) {
+cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStream_t s) {
     if (n_items <= 0) return cudaSuccess;
-    if (p.G > 8)
-        decode_kernel<true><<<n_items, kWarps * 32, kSmemBytes, s>>>(p);
-    else
-        decode_kernel<false><<<n_items, kWarps * 32, kSmemBytes, s>>>(p);
+    if (warps == 8) {
+        if (p.G > 8)
+            decode_kernel<true, 8><<<n_items, 256, 8 * kWarpSmem, s>>>(p);
+        else
+            decode_kernel<false, 8><<<n_items, 256, 8 * kWarpSmem, s>>>(p);
+    } else {
+        if (p.G > 8)
+            decode_kernel<true, 4><<<n_items, 128, 4 * kWarpSmem, s>>>(p);
+        else
+            decode_kernel<false, 4><<<n_items, 128, 4 * kWarpSmem, s>>>(p);
+    }
     count_launch();
     return cudaGetLastError();
 }

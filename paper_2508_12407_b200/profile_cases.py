@@ -1,0 +1,75 @@
+"""Small, self-contained launches of each kernel for profiling under ncu.
+
+    python -m paper_2508_12407_b200.profile_cases --case decode_r [--n 32768] [--batch 1] [--reps 3]
+
+Each case holds well under a few GB on the device and its inputs exceed the 126 MB L2, so a
+capture of one to three launches ends by itself and its DRAM counters are meaningful.
+Cases: decode_r (retrieval decode), decode_s (streaming decode), prefill_r, prefill_s,
+append (decode-time append), mixed (mixed-head decode layer).
+"""
+from __future__ import annotations
+
+import argparse
+
+import numpy as np
+import torch
+
+from . import binding, build
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--case", required=True,
+                    choices=["decode_r", "decode_s", "prefill_r", "prefill_s", "append", "mixed"])
+    ap.add_argument("--n", type=int, default=32768, help="context length (decode) or chunk length (prefill)")
+    ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--layers", type=int, default=2)
+    ap.add_argument("--reps", type=int, default=3)
+    ap.add_argument("--recent", type=int, default=256)
+    args = ap.parse_args()
+    build.build()
+    binding.load()
+    dev = torch.device("cuda:0")
+    g = torch.Generator(device=dev)
+    g.manual_seed(7)
+    Hq, Hkv, D, S, W = 32, 8, 128, 128, args.recent
+    B, N, L = args.batch, args.n, args.layers
+
+    def randn(*shape):
+        return torch.randn(*shape, device=dev, generator=g, dtype=torch.float32).to(torch.bfloat16)
+
+    kind = 1 if args.case in ("decode_r", "prefill_r", "append") else 0
+    kvk = None
+    if args.case == "mixed":
+        kvk = np.tile(np.array([1, 0, 1, 0, 0, 1, 1, 0], dtype=np.uint8), (L, 1))
+    cache = binding.ZigzagCache(L, B, Hq, Hkv, S, W, [kind] * L, [N + 64] * B, max(B * N, B),
+                                kvhead_is_retrieval=kvk)
+    if args.case in ("prefill_r", "prefill_s"):
+        q, k, v = randn(B * N, Hq, D), randn(B * N, Hkv, D), randn(B * N, Hkv, D)
+        out = torch.empty_like(q)
+        for _ in range(args.reps):
+            for l in range(L):
+                cache.prefill_attn(l, q, k, v, out, [N] * B)
+    else:
+        CH = 8192
+        for l in range(L):
+            done = 0
+            while done < N:
+                c = min(CH, N - done)
+                cache.kv_append(l, randn(B * c, Hkv, D), randn(B * c, Hkv, D), [c] * B)
+                done += c
+        q, k, v = randn(B, Hq, D), randn(B, Hkv, D), randn(B, Hkv, D)
+        out = torch.empty_like(q)
+        for _ in range(args.reps):
+            for l in range(L):
+                if args.case == "append":
+                    cache.kv_append(l, k, v, [1] * B)
+                else:
+                    cache.decode_attn(l, q, out)
+    torch.cuda.synchronize()
+    assert cache.last_status() == 0
+    print("done", args.case, "launches", binding.launch_count())
+
+
+if __name__ == "__main__":
+    main()
