@@ -186,6 +186,39 @@ int zz_get_last_status(zz_cache_t* cache, void* stream);
 int zz_profile_enable(int period);
 int zz_profile_read(int kind, int64_t* launches, double* total_ms, int reset);
 
+/* Decode attention without any workspace from the caller (the paper has no counterpart: this
+ * is a deployment convenience, not part of the method).
+ *
+ * For callers that cannot allocate device memory -- a server that has given the whole device
+ * to its own pool, a plug-in whose host forbids allocations after start-up, code that may run
+ * while a stream is being captured -- and therefore cannot hand the library a workspace.  The
+ * scratch the split-sequence decode kernel needs (partial outputs, their softmax statistics,
+ * arrival counters, the device copy of the lengths) lives in a fixed array of about 2.1 MB
+ * inside the library's device image; every GPU that loads the library holds it until the
+ * process exits.  The call itself never calls cudaMalloc, cudaFree or any allocating routine.
+ *
+ * Computes, for each sequence b, full (retrieval) attention of one query token over the first
+ * h_len[b] rows of the caller's stores:
+ *   d_q, d_out  [batch, n_q_heads, 128] bf16 (device)
+ *   d_k, d_v    [batch, n_kv_heads, capacity, 128] bf16 (device), row j = token j
+ *   h_len       [batch] int32 (host), 1 <= h_len[b] <= capacity
+ * Limits, fixed by the size of the array: batch <= 16 and batch * n_q_heads <= 64; anything
+ * larger is refused with ZZ_ERR_WORKSPACE before anything is launched (the limits can be read
+ * with zz_decode_attn_static_limits).  Group size and head_dim rules are the library's usual ones.
+ *
+ * The first call on a device looks up the array's device address (and opts the kernel into its
+ * shared-memory size); make that first call outside any stream capture.  All calls, from every
+ * thread and stream, share the one array per device: it keeps the previous call's contents (the
+ * call clears the counters it needs at zero itself), and two calls whose kernels may overlap on
+ * the GPU race on it -- issue them on one stream, or order them yourself.  Asynchronous on
+ * `stream`; h_len may be reused as soon as the call returns if it is pageable memory, and after
+ * the stream reaches the copy if it is pinned. */
+int zz_decode_attn_static(const void* d_q, const void* d_k, const void* d_v, void* d_out,
+                          const int32_t* h_len, int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
+                          int32_t capacity, float softmax_scale, void* stream);
+int zz_decode_attn_static_limits(int32_t* max_batch, int32_t* max_batch_times_q_heads,
+                                 size_t* scratch_bytes);
+
 /* Number of kernels this library has launched since it was loaded (all handles). */
 int64_t zz_launch_count(void);
 

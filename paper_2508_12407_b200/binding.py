@@ -81,6 +81,9 @@ SYMBOLS = {
     "zz_cache_export": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, ctypes.POINTER(ctypes.c_int32), _vp]),
     "zz_cache_import": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp]),
     "zz_get_last_status": (_i32, [_vp, _vp]),
+    "zz_decode_attn_static": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, ctypes.c_float, _vp]),
+    "zz_decode_attn_static_limits": (_i32, [ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
+                                            ctypes.POINTER(_sz)]),
 }
 
 
@@ -298,6 +301,28 @@ class ZigzagCache:
 
     def last_status(self, stream=None) -> int:
         return int(self._lib.zz_get_last_status(self._h, _stream_ptr(stream)))
+
+
+def decode_attn_static(q, k, v, out, lens, softmax_scale: Optional[float] = None, stream=None) -> None:
+    """Workspace-free decode attention for callers that cannot allocate device memory.
+
+    q/out [batch, n_q_heads, 128], k/v [batch, n_kv_heads, capacity, 128] (device, bf16),
+    lens: host integers.  The scratch is a fixed array inside the library, shared by all calls:
+    keep calls that might overlap on the GPU on one stream."""
+    B, Hq, D = q.shape
+    _, Hkv, cap, _ = k.shape
+    hl = np.ascontiguousarray(np.asarray(lens, dtype=np.int32))
+    assert hl.shape == (B,) and v.shape == k.shape and out.shape == q.shape
+    scale = float(softmax_scale) if softmax_scale is not None else 1.0 / float(np.sqrt(D))
+    _check(load().zz_decode_attn_static(_dptr(q), _dptr(k), _dptr(v), _dptr(out), _np_ptr(hl), B, Hq, Hkv,
+                                        cap, scale, _stream_ptr(stream)), "zz_decode_attn_static")
+
+
+def decode_attn_static_limits():
+    mb, mr, sb = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_size_t(0)
+    _check(load().zz_decode_attn_static_limits(ctypes.byref(mb), ctypes.byref(mr), ctypes.byref(sb)),
+           "zz_decode_attn_static_limits")
+    return int(mb.value), int(mr.value), int(sb.value)
 
 
 def bf16_bits_to_tensor(bits: np.ndarray, device="cuda:0"):
