@@ -36,6 +36,10 @@ constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 1024;
 constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr uint32_t kAbortPolls = 1u << 10;
 constexpr float kRescaleThreshold = 8.f;    // log2 units of slack before O is rescaled
+#ifndef ZZ_POLY_EVERY
+#define ZZ_POLY_EVERY 4
+#endif
+constexpr int kPolyEvery = ZZ_POLY_EVERY;   // one pair in kPolyEvery takes the polynomial exp2 (>= 17: none)
 
 // instruction descriptor: fp32 accumulate, bf16 A and B, M = 128, N = 128
 constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
@@ -76,7 +80,9 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait.  Returns false (after flagging the error) if the phase never completed.
-__device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Shared* sh, int* status) {
+// The first probe is inlined: a wait on a phase that has already completed costs one
+// try_wait, and only a real wait enters the polling loop.
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, Shared* sh, int* status) {
     const uint32_t limit = (*(volatile int*)&sh->abort_flag) ? kAbortPolls : kMaxPolls;
     for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try(bar, parity)) return true;
@@ -85,6 +91,10 @@ __device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Shared* s
     *(volatile int*)&sh->abort_flag = 1;
     atomicExch(status, ZZ_ERR_TIMEOUT);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Shared* sh, int* status) {
+    if (mbar_try(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, sh, status);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
@@ -180,6 +190,45 @@ __device__ __forceinline__ float fast_exp2(float x) {
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// two fp32 lanes per instruction (packed FMA / ADD of sm_100)
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
+    float2 d;
+    asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "mov.b64 rc, {%6, %7};\n\tfma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d.x), "=f"(d.y)
+        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+    return d;
+}
+__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+    float2 d;
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d.x), "=f"(d.y)
+        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
+}
+// 2^x for a pair of finite x on the FMA pipe instead of the MUFU: x = n + f with n = round(x)
+// (taken from the low mantissa bits of x + 1.5 * 2^23) and f in [-0.5, 0.5]; 2^f by a cubic
+// fitted to minimise the relative error on that interval (7.5e-5, far below the bf16 rounding of
+// the probabilities); n goes straight into the exponent field.
+__device__ __forceinline__ float2 exp2_poly2(float2 x) {
+    const float kMagic = 12582912.f;
+    const float2 t = add2(x, make_float2(kMagic, kMagic));
+    const float2 r = add2(t, make_float2(-kMagic, -kMagic));
+    const float2 f = fma2(r, make_float2(-1.f, -1.f), x);
+    float2 p = fma2(make_float2(0.055171408f, 0.055171408f), f, make_float2(0.24261075f, 0.24261075f));
+    p = fma2(p, f, make_float2(0.69326097f, 0.69326097f));
+    p = fma2(p, f, make_float2(0.99992812f, 0.99992812f));
+    float2 o;
+    o.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
+    o.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
+    return o;
 }
 
 // Which KV tiles a query tile visits, in order: store tiles, then chunk tiles (sink tiles of
@@ -322,6 +371,12 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
         // ================= MMA issuer =================
         if (lane == 0) {
             const int n_act = active1 ? 2 : 1;
+            // Descriptors differ only in the 14-bit start-address field (bytes >> 4), which never
+            // carries out of that field for shared-memory addresses, so each one is base + offset.
+            const uint64_t dq = make_desc(sm_q, 16, 1024);          // Q tile 0, K-major
+            const uint64_t dk = make_desc(sm_kv, 16, 1024);         // K tile in stage 0, K-major
+            const uint64_t dv = make_desc(sm_kv, kSubBytes, 1024);  // V tile in stage 0, MN-major
+            constexpr uint32_t kTile16 = kTileBytes >> 4;
             mbar_wait(&sh.q_full, 0, &sh, p.status);
             mbar_wait(&sh.kv_full[0], 0, &sh, p.status);
             tc_fence_after();
@@ -329,9 +384,8 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
             for (int t = 0; t < n_act; ++t) {
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t off = (kk >> 2) * kSubBytes + (kk & 3) * 32;
-                    mma_ss(tmem + t * 256, make_desc(sm_q + t * kTileBytes + off, 16, 1024),
-                           make_desc(sm_kv + off, 16, 1024), kIdescQK, kk > 0);
+                    const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
+                    mma_ss(tmem + t * 256, dq + t * kTile16 + off16, dk + off16, kIdescQK, kk > 0);
                 }
                 mma_commit(&sh.s_full[t]);
             }
@@ -340,26 +394,30 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                 const int uv = 2 * j + 1, uk = 2 * j + 2;
                 const int sv = uv % kStages, sk = uk % kStages;
                 const bool more = (j + 1) < n_tiles;
+                const uint64_t dvj = dv + sv * kTile16, dkj = dk + sk * kTile16;
                 mbar_wait(&sh.kv_full[sv], (uv / kStages) & 1, &sh, p.status);
                 if (more) mbar_wait(&sh.kv_full[sk], (uk / kStages) & 1, &sh, p.status);
                 for (int t = 0; t < n_act; ++t) {
                     mbar_wait(&sh.p_full[t], j & 1, &sh, p.status);
                     tc_fence_after();
                     // O_t (+)= P_t V_j
+                    const uint32_t t_st = tmem + t * 256;
+                    if (j > 0) {
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        mma_ts(tmem + t * 256 + 128, tmem + t * 256 + kk * 8,
-                               make_desc(sm_kv + sv * kTileBytes + kk * 2048, kSubBytes, 1024), kIdescPV,
-                               (j > 0) || (kk > 0));
+                        for (int kk = 0; kk < 8; ++kk)
+                            mma_ts(t_st + 128, t_st + kk * 8, dvj + kk * (2048 >> 4), kIdescPV, true);
+                    } else {
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk)
+                            mma_ts(t_st + 128, t_st + kk * 8, dvj + kk * (2048 >> 4), kIdescPV, kk > 0);
                     }
                     if (t == n_act - 1) mma_commit(&sh.kv_empty[sv]);
                     if (more) {
                         // S_t = Q_t K_{j+1}^T
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
-                            const uint32_t off = (kk >> 2) * kSubBytes + (kk & 3) * 32;
-                            mma_ss(tmem + t * 256, make_desc(sm_q + t * kTileBytes + off, 16, 1024),
-                                   make_desc(sm_kv + sk * kTileBytes + off, 16, 1024), kIdescQK, kk > 0);
+                            const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
+                            mma_ss(t_st, dq + t * kTile16 + off16, dkj + off16, kIdescQK, kk > 0);
                         }
                         mma_commit(&sh.s_full[t]);
                         if (t == n_act - 1) mma_commit(&sh.kv_empty[sk]);
@@ -394,10 +452,13 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                 tmem_wait_ld();
 
                 // ---- visibility ----------------------------------------------------------------
+                // tile_masked: some entry of this 128 x 128 tile may be invisible (uniform over the CTA)
+                bool tile_masked = true;
                 if (p.kind == ZZ_KIND_RETRIEVAL) {
                     int lim = 128;                                    // columns [0, lim) are visible
                     if (!is_chunk) lim = plan.n_occ - start;          // rows past the store's length
                     else lim = rr - start + 1;                        // causal inside the chunk
+                    tile_masked = is_chunk ? (start + 127 > r0) : (plan.n_occ - start < 128);
                     if (lim < 128) {
 #pragma unroll
                         for (int c = 0; c < 128; ++c)
@@ -427,10 +488,18 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                 }
 
                 // ---- running maximum, lazily applied ---------------------------------------------
-                float mx = s[0];
+                float mx;
+                {
+                    float mc[4];
 #pragma unroll
-                for (int c = 1; c < 128; ++c) mx = fmaxf(mx, s[c]);
-                mx *= sc;
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        float a = s[q4 * 32];
+#pragma unroll
+                        for (int i = 1; i < 31; i += 2) a = max3(a, s[q4 * 32 + i], s[q4 * 32 + i + 1]);
+                        mc[q4] = fmaxf(a, s[q4 * 32 + 31]);
+                    }
+                    mx = fmaxf(max3(mc[0], mc[1], mc[2]), mc[3]) * sc;
+                }
                 float alpha = 1.f;
                 bool bump = false;
                 if (mx > m_used + kRescaleThreshold || (m_used == -INFINITY && mx > -INFINITY)) {
@@ -451,20 +520,43 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                         tmem_st32(t_o + c * 32, o);
                     }
                 }
+                // ---- probabilities: p = 2^(s * scale - m), bf16 into tensor memory, fp32 row sum ----
+                // The MUFU evaluates 16 exponentials per clock and SM, which for a 128 x 128 tile is as
+                // long as its two MMAs; on tiles without masked (-inf) entries every kPolyEvery-th
+                // pair is therefore evaluated by a polynomial on the FMA pipe instead.
                 const float msub = (m_used == -INFINITY) ? 0.f : m_used;
-                float psum = 0.f;
+                const float2 sc2 = make_float2(sc, sc), nm2 = make_float2(-msub, -msub);
+                float2 ps2 = make_float2(0.f, 0.f);
+                if (tile_masked) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t pk[16];
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t pk[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float p0 = fast_exp2(fmaf(s[c * 32 + 2 * i], sc, -msub));
-                        const float p1 = fast_exp2(fmaf(s[c * 32 + 2 * i + 1], sc, -msub));
-                        psum += p0 + p1;
-                        pk[i] = pack_bf16(p0, p1);
+                        for (int i = 0; i < 16; ++i) {
+                            const float2 x = fma2(make_float2(s[c * 32 + 2 * i], s[c * 32 + 2 * i + 1]), sc2, nm2);
+                            const float2 e = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+                            ps2 = add2(ps2, e);
+                            pk[i] = pack_bf16(e.x, e.y);
+                        }
+                        tmem_st16(t_s + c * 16, pk);
                     }
-                    tmem_st16(t_s + c * 16, pk);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const float2 x = fma2(make_float2(s[c * 32 + 2 * i], s[c * 32 + 2 * i + 1]), sc2, nm2);
+                            const float2 e = ((i % kPolyEvery) == kPolyEvery - 1)
+                                                 ? exp2_poly2(x)
+                                                 : make_float2(fast_exp2(x.x), fast_exp2(x.y));
+                            ps2 = add2(ps2, e);
+                            pk[i] = pack_bf16(e.x, e.y);
+                        }
+                        tmem_st16(t_s + c * 16, pk);
+                    }
                 }
+                const float psum = ps2.x + ps2.y;
                 l_run += psum;
                 tmem_wait_st();
                 tc_fence_before();
