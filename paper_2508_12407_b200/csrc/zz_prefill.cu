@@ -10,10 +10,12 @@
 //
 // CTA = one 128-token query tile x two query heads of the same KV head, so each K/V tile is
 // fetched once for two score tiles and the two tiles ping-pong on the tensor pipe:
-//   warp 0      TMA producer (one elected lane)
-//   warp 1      MMA issuer   (one elected lane)
-//   warps 2-5   softmax / correction / epilogue of tile 0 (one thread per query row)
-//   warps 6-9   the same for tile 1
+//   warps 0-3   softmax / correction / epilogue of tile 0 (one thread per query row)
+//   warps 4-7   the same for tile 1
+//   warp 8      TMA producer (one elected lane)
+//   warp 9      MMA issuer   (one elected lane)
+//   warps 10-11 idle: they only complete the third warpgroup, which hands most of its registers
+//               to the two softmax warpgroups (setmaxnreg)
 // Tensor memory (512 columns): tile t has S_t at column 256 t (128 fp32 columns; the bf16
 // probabilities P_t overwrite its first 64 columns and feed the PV MMA as the A operand from
 // tensor memory) and O_t at column 256 t + 128.
@@ -31,7 +33,9 @@ constexpr int kTile = 128;
 constexpr int kSubBytes = 128 * 128;        // [128 rows][64 bf16] sub-tile, 128-byte swizzled
 constexpr int kTileBytes = 2 * kSubBytes;   // a full [128][128] bf16 tile
 constexpr int kStages = 4;                  // ring of K and V tiles (K_0, V_0, K_1, V_1, ...)
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;                // three warpgroups: softmax tile 0, softmax tile 1, TMA + MMA
+constexpr int kWarpTma = 8, kWarpMma = 9;
+constexpr int kRegsSoftmax = 224, kRegsAux = 56;   // 224 * 256 + 56 * 128 <= 65536 registers
 constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 1024;
 constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr uint32_t kAbortPolls = 1u << 10;
@@ -82,7 +86,7 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
 // Bounded wait.  Returns false (after flagging the error) if the phase never completed.
 // The first probe is inlined: a wait on a phase that has already completed costs one
 // try_wait, and only a real wait enters the polling loop.
-__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, Shared* sh, int* status) {
+__device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, Shared* sh, int* status) {
     const uint32_t limit = (*(volatile int*)&sh->abort_flag) ? kAbortPolls : kMaxPolls;
     for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try(bar, parity)) return true;
@@ -231,6 +235,13 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x) {
     return o;
 }
 
+// bits i of a 32-bit word that stand for columns base + i inside [lo, hi]
+__device__ __forceinline__ uint32_t range_bits(int lo, int hi, int base) {
+    const int a = max(lo - base, 0), b = min(hi - base, 31);
+    if (a > b) return 0u;
+    return (0xffffffffu >> (31 - b)) & (0xffffffffu << a);
+}
+
 // Which KV tiles a query tile visits, in order: store tiles, then chunk tiles (sink tiles of
 // the chunk that lie before the band, then the band up to the diagonal).
 struct TilePlan {
@@ -320,7 +331,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 0) {
+    if (warp == kWarpTma) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&sh.tmem_base))
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -330,7 +341,11 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
     tc_fence_after();
     const uint32_t tmem = *(volatile uint32_t*)&sh.tmem_base;
 
-    if (warp == 0) {
+    // Registers move from the TMA/MMA warpgroup (which needs few) to the softmax warpgroups, whose
+    // threads each hold a 128-column row of scores.
+    if (warp >= 8) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsAux));
+      if (warp == kWarpTma) {
         // ================= TMA producer =================
         if (lane == 0) {
             const SeqDesc sd = p.desc[b];
@@ -367,7 +382,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                 }
             }
         }
-    } else if (warp == 1) {
+      } else if (warp == kWarpMma) {
         // ================= MMA issuer =================
         if (lane == 0) {
             const int n_act = active1 ? 2 : 1;
@@ -426,9 +441,11 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
             }
             mma_commit(&sh.o_full);
         }
+      }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
         // ================= softmax / correction / epilogue =================
-        const int t = (warp - 2) >> 2;                  // which of the two tiles
+        const int t = warp >> 2;                        // which of the two tiles
         if (t == 0 || active1) {
             const int quarter = warp & 3;               // tensor-memory lanes this warp may touch
             const int r = quarter * 32 + lane;          // query row inside the tile
@@ -452,39 +469,47 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                 tmem_wait_ld();
 
                 // ---- visibility ----------------------------------------------------------------
-                // tile_masked: some entry of this 128 x 128 tile may be invisible (uniform over the CTA)
+                // tile_masked: some entry of this 128 x 128 tile may be invisible (uniform over the
+                // CTA); vis[w] bit i: column 32 w + i is visible to this thread's row
                 bool tile_masked = true;
-                if (p.kind == ZZ_KIND_RETRIEVAL) {
-                    int lim = 128;                                    // columns [0, lim) are visible
-                    if (!is_chunk) lim = plan.n_occ - start;          // rows past the store's length
-                    else lim = rr - start + 1;                        // causal inside the chunk
+                if (p.kind == ZZ_KIND_RETRIEVAL)
                     tile_masked = is_chunk ? (start + 127 > r0) : (plan.n_occ - start < 128);
-                    if (lim < 128) {
+                if (tile_masked) {
+                    uint32_t vis[4];
+                    if (p.kind == ZZ_KIND_RETRIEVAL) {
+                        // store rows past the store's length; causal inside the chunk
+                        const int lim = is_chunk ? (rr - start + 1) : (plan.n_occ - start);
 #pragma unroll
-                        for (int c = 0; c < 128; ++c)
-                            if (c >= lim) s[c] = -INFINITY;
-                    }
-                } else if (!is_chunk) {
-                    const int tq = P + rr;
+                        for (int w = 0; w < 4; ++w) vis[w] = range_bits(0, lim - 1, 32 * w);
+                    } else if (!is_chunk) {
+                        const int tq = P + rr;
 #pragma unroll
-                    for (int c = 0; c < 128; ++c) {
-                        const int idx = start + c;
-                        bool ok = idx < plan.n_occ;
-                        if (ok) {
-                            const int pp = pos[idx];
-                            ok = (pp < p.S) || (tq - pp < p.W);
+                        for (int w = 0; w < 4; ++w) {
+                            uint32_t m = 0;
+#pragma unroll 4
+                            for (int i = 0; i < 32; ++i) {
+                                const int idx = start + 32 * w + i;
+                                bool ok = idx < plan.n_occ;
+                                if (ok) {
+                                    const int pp = pos[idx];
+                                    ok = (pp < p.S) || (tq - pp < p.W);
+                                }
+                                m |= (ok ? 1u : 0u) << i;
+                            }
+                            vis[w] = m;
                         }
-                        if (!ok) s[c] = -INFINITY;
-                    }
-                } else {
-                    const int c_hi = rr - start;                      // causal
-                    const int c_lo = rr - p.W + 1 - start;            // window
-                    const int c_sink = p.S - P - start;               // chunk tokens that are sinks
+                    } else {
+                        const int c_hi = rr - start;                      // causal
+                        const int c_lo = rr - p.W + 1 - start;            // window
+                        const int c_sink = p.S - P - start;               // chunk tokens that are sinks
 #pragma unroll
-                    for (int c = 0; c < 128; ++c) {
-                        const bool ok = (c <= c_hi) && ((c >= c_lo) || (c < c_sink));
-                        if (!ok) s[c] = -INFINITY;
+                        for (int w = 0; w < 4; ++w)
+                            vis[w] = range_bits(0, c_hi, 32 * w) &
+                                     (range_bits(c_lo, 127, 32 * w) | range_bits(0, c_sink - 1, 32 * w));
                     }
+#pragma unroll
+                    for (int c = 0; c < 128; ++c)
+                        if (!((vis[c >> 5] >> (c & 31)) & 1u)) s[c] = -INFINITY;
                 }
 
                 // ---- running maximum, lazily applied ---------------------------------------------
@@ -592,7 +617,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) {
+    if (warp == kWarpTma) {
         // every TMA load this CTA issued has been consumed (the MMA warp waited on each full
         // barrier), and every MMA has completed (o_full); tensor memory can go back
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
