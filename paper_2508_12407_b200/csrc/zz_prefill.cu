@@ -83,6 +83,19 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// Non-blocking probe of a phase (try_wait may suspend the thread for a while when the phase is
+// still open; a probe must not).
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 // Bounded wait.  Returns false (after flagging the error) if the phase never completed.
 // The first probe is inlined: a wait on a phase that has already completed costs one
 // try_wait, and only a real wait enters the polling loop.
@@ -126,18 +139,24 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
     return d;
 }
 
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool acc) {
+// Descriptors travel as (low word, high word): only the low word (start address >> 4 in its 14
+// low bits) changes between the MMAs of a tile, so stepping one costs a single 32-bit add.
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t ab_hi_a,
+                                       uint32_t ab_hi_b, uint32_t idesc, bool acc) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"((uint32_t)acc)
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(ab_hi_a), "r"(b_lo), "r"(ab_hi_b), "r"(idesc), "r"((uint32_t)acc)
         : "memory");
 }
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, bool acc) {
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
+                                       uint32_t idesc, bool acc) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"((uint32_t)acc)
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"((uint32_t)acc)
         : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
@@ -386,11 +405,11 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
         // ================= MMA issuer =================
         if (lane == 0) {
             const int n_act = active1 ? 2 : 1;
-            // Descriptors differ only in the 14-bit start-address field (bytes >> 4), which never
-            // carries out of that field for shared-memory addresses, so each one is base + offset.
             const uint64_t dq = make_desc(sm_q, 16, 1024);          // Q tile 0, K-major
             const uint64_t dk = make_desc(sm_kv, 16, 1024);         // K tile in stage 0, K-major
             const uint64_t dv = make_desc(sm_kv, kSubBytes, 1024);  // V tile in stage 0, MN-major
+            const uint32_t dq_lo = (uint32_t)dq, dk_lo = (uint32_t)dk, dv_lo = (uint32_t)dv;
+            const uint32_t dkm_hi = (uint32_t)(dq >> 32), dv_hi = (uint32_t)(dv >> 32);
             constexpr uint32_t kTile16 = kTileBytes >> 4;
             mbar_wait(&sh.q_full, 0, &sh, p.status);
             mbar_wait(&sh.kv_full[0], 0, &sh, p.status);
@@ -400,42 +419,71 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
                     const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
-                    mma_ss(tmem + t * 256, dq + t * kTile16 + off16, dk + off16, kIdescQK, kk > 0);
+                    mma_ss(tmem + t * 256, dq_lo + t * kTile16 + off16, dk_lo + off16, dkm_hi, dkm_hi, kIdescQK,
+                           kk > 0);
                 }
                 mma_commit(&sh.s_full[t]);
             }
             mma_commit(&sh.kv_empty[0]);
+            // The thread that issues tcgen05.mma is held at each one until the tensor pipe has room, so
+            // whatever it does between two tiles leaves the pipe idle.  The barriers of the next tile
+            // (K/V stages, the other tile's P) are therefore probed two MMAs before the current
+            // tile's last one; the probe's latency then overlaps those MMAs, and the blocking wait is
+            // only entered when a probe came back negative.
+            bool ok_v = mbar_test(&sh.kv_full[1 % kStages], 0);
+            bool ok_k = (n_tiles > 1) ? mbar_test(&sh.kv_full[2 % kStages], 0) : true;
+            bool ok_p = mbar_test(&sh.p_full[0], 0);
             for (int j = 0; j < n_tiles; ++j) {
                 const int uv = 2 * j + 1, uk = 2 * j + 2;
                 const int sv = uv % kStages, sk = uk % kStages;
                 const bool more = (j + 1) < n_tiles;
-                const uint64_t dvj = dv + sv * kTile16, dkj = dk + sk * kTile16;
-                mbar_wait(&sh.kv_full[sv], (uv / kStages) & 1, &sh, p.status);
-                if (more) mbar_wait(&sh.kv_full[sk], (uk / kStages) & 1, &sh, p.status);
+                const uint32_t dvj = dv_lo + sv * kTile16, dkj = dk_lo + sk * kTile16;
+                if (!ok_v) mbar_wait(&sh.kv_full[sv], (uv / kStages) & 1, &sh, p.status);
+                if (!ok_k) mbar_wait(&sh.kv_full[sk], (uk / kStages) & 1, &sh, p.status);
                 for (int t = 0; t < n_act; ++t) {
-                    mbar_wait(&sh.p_full[t], j & 1, &sh, p.status);
+                    if (!ok_p) mbar_wait(&sh.p_full[t], j & 1, &sh, p.status);
                     tc_fence_after();
-                    // O_t (+)= P_t V_j
                     const uint32_t t_st = tmem + t * 256;
+                    const uint32_t dqt = dq_lo + t * kTile16;
+                    const bool last_of_iter = (t == n_act - 1);
+                    // probes for what is issued after this tile's MMAs
+                    auto probe_next = [&]() {
+                        if (!last_of_iter) {
+                            ok_p = mbar_test(&sh.p_full[1], j & 1);
+                        } else if (more) {
+                            const int uv2 = uv + 2, uk2 = uk + 2;
+                            ok_v = mbar_test(&sh.kv_full[uv2 % kStages], (uv2 / kStages) & 1);
+                            ok_k = (j + 2 < n_tiles) ? mbar_test(&sh.kv_full[uk2 % kStages], (uk2 / kStages) & 1) : true;
+                            ok_p = mbar_test(&sh.p_full[0], (j + 1) & 1);
+                        }
+                    };
+                    // O_t (+)= P_t V_j
                     if (j > 0) {
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk)
-                            mma_ts(t_st + 128, t_st + kk * 8, dvj + kk * (2048 >> 4), kIdescPV, true);
+                        for (int kk = 0; kk < 8; ++kk) {
+                            if (kk == 6 && !more) probe_next();
+                            mma_ts(t_st + 128, t_st + kk * 8, dvj + kk * (2048 >> 4), dv_hi, kIdescPV, true);
+                        }
                     } else {
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk)
-                            mma_ts(t_st + 128, t_st + kk * 8, dvj + kk * (2048 >> 4), kIdescPV, kk > 0);
+                        for (int kk = 0; kk < 8; ++kk) {
+                            if (kk == 6 && !more) probe_next();
+                            mma_ts(t_st + 128, t_st + kk * 8, dvj + kk * (2048 >> 4), dv_hi, kIdescPV, kk > 0);
+                        }
                     }
-                    if (t == n_act - 1) mma_commit(&sh.kv_empty[sv]);
+                    if (last_of_iter) mma_commit(&sh.kv_empty[sv]);
                     if (more) {
                         // S_t = Q_t K_{j+1}^T
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
+                            if (kk == 6) probe_next();
                             const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
-                            mma_ss(t_st, dq + t * kTile16 + off16, dkj + off16, kIdescQK, kk > 0);
+                            mma_ss(t_st, dqt + off16, dkj + off16, dkm_hi, dkm_hi, kIdescQK, kk > 0);
                         }
+                    }
+                    if (more) {
                         mma_commit(&sh.s_full[t]);
-                        if (t == n_act - 1) mma_commit(&sh.kv_empty[sk]);
+                        if (last_of_iter) mma_commit(&sh.kv_empty[sk]);
                     }
                 }
             }
@@ -512,76 +560,93 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                         if (!((vis[c >> 5] >> (c & 31)) & 1u)) s[c] = -INFINITY;
                 }
 
-                // ---- running maximum, lazily applied ---------------------------------------------
-                float mx;
-                {
-                    float mc[4];
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        float a = s[q4 * 32];
-#pragma unroll
-                        for (int i = 1; i < 31; i += 2) a = max3(a, s[q4 * 32 + i], s[q4 * 32 + i + 1]);
-                        mc[q4] = fmaxf(a, s[q4 * 32 + 31]);
-                    }
-                    mx = fmaxf(max3(mc[0], mc[1], mc[2]), mc[3]) * sc;
-                }
-                float alpha = 1.f;
-                bool bump = false;
-                if (mx > m_used + kRescaleThreshold || (m_used == -INFINITY && mx > -INFINITY)) {
-                    alpha = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - mx);
-                    m_used = mx;
-                    l_run *= alpha;
-                    bump = true;
-                }
-                if (j > 0 && __any_sync(0xffffffffu, bump)) {
-                    // PV of the previous tile has completed (its commit precedes s_full), so O is stable
-                    float o[32];
-#pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        tmem_ld32(t_o + c * 32, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] *= alpha;
-                        tmem_st32(t_o + c * 32, o);
-                    }
-                }
-                // ---- probabilities: p = 2^(s * scale - m), bf16 into tensor memory, fp32 row sum ----
+                // ---- probabilities p = 2^(s * scale - m) as bf16 into tensor memory, fp32 row sum ----
+                // m is any upper estimate of the row maximum that keeps 2^(s * scale - m) finite, so the
+                // exponentials do not wait for this tile's maximum: they are taken against the running
+                // m, the tile's maximum is reduced alongside them (other pipe, no dependency), and only if
+                // it exceeds m by more than the threshold is m raised, O rescaled and the tile redone.
                 // The MUFU evaluates 16 exponentials per clock and SM, which for a 128 x 128 tile is as
                 // long as its two MMAs; on tiles without masked (-inf) entries every kPolyEvery-th
                 // pair is therefore evaluated by a polynomial on the FMA pipe instead.
-                const float msub = (m_used == -INFINITY) ? 0.f : m_used;
-                const float2 sc2 = make_float2(sc, sc), nm2 = make_float2(-msub, -msub);
-                float2 ps2 = make_float2(0.f, 0.f);
-                if (tile_masked) {
+                float psum = 0.f;
+#pragma unroll 1
+                for (int attempt = 0; attempt < 2; ++attempt) {
+                    const bool do_exp = (attempt == 1) || (j > 0);
+                    float mc[4];
+                    if (do_exp) {
+                        const float msub = (m_used == -INFINITY) ? 0.f : m_used;
+                        const float2 sc2 = make_float2(sc, sc), nm2 = make_float2(-msub, -msub);
+                        float2 ps2 = make_float2(0.f, 0.f);
+                        if (tile_masked) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t pk[16];
+                            for (int c = 0; c < 4; ++c) {
+                                uint32_t pk[16];
+                                float a = s[c * 32];
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const float2 x = fma2(make_float2(s[c * 32 + 2 * i], s[c * 32 + 2 * i + 1]), sc2, nm2);
-                            const float2 e = make_float2(fast_exp2(x.x), fast_exp2(x.y));
-                            ps2 = add2(ps2, e);
-                            pk[i] = pack_bf16(e.x, e.y);
+                                for (int i = 0; i < 16; ++i) {
+                                    const float s0 = s[c * 32 + 2 * i], s1 = s[c * 32 + 2 * i + 1];
+                                    a = max3(a, s0, s1);
+                                    const float2 x = fma2(make_float2(s0, s1), sc2, nm2);
+                                    const float2 e = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+                                    ps2 = add2(ps2, e);
+                                    pk[i] = pack_bf16(e.x, e.y);
+                                }
+                                mc[c] = a;
+                                tmem_st16(t_s + c * 16, pk);
+                            }
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                uint32_t pk[16];
+                                float a = s[c * 32];
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) {
+                                    const float s0 = s[c * 32 + 2 * i], s1 = s[c * 32 + 2 * i + 1];
+                                    a = max3(a, s0, s1);
+                                    const float2 x = fma2(make_float2(s0, s1), sc2, nm2);
+                                    const float2 e = ((i % kPolyEvery) == kPolyEvery - 1)
+                                                         ? exp2_poly2(x)
+                                                         : make_float2(fast_exp2(x.x), fast_exp2(x.y));
+                                    ps2 = add2(ps2, e);
+                                    pk[i] = pack_bf16(e.x, e.y);
+                                }
+                                mc[c] = a;
+                                tmem_st16(t_s + c * 16, pk);
+                            }
                         }
-                        tmem_st16(t_s + c * 16, pk);
+                        psum = ps2.x + ps2.y;
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            float a = s[c * 32];
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) a = max3(a, s[c * 32 + 2 * i], s[c * 32 + 2 * i + 1]);
+                            mc[c] = a;
+                        }
                     }
-                } else {
+                    if (attempt == 1) break;
+                    const float mx = fmaxf(max3(mc[0], mc[1], mc[2]), mc[3]) * sc;
+                    const bool bump = mx > m_used + kRescaleThreshold || (m_used == -INFINITY && mx > -INFINITY);
+                    if (do_exp && !__any_sync(0xffffffffu, bump)) break;
+                    float alpha = 1.f;
+                    if (bump) {
+                        alpha = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - mx);
+                        m_used = mx;
+                        l_run *= alpha;
+                    }
+                    if (j > 0) {
+                        // PV of the previous tile has completed (its commit precedes s_full), so O is stable
+                        float o[32];
+#pragma unroll 1
+                        for (int c = 0; c < 4; ++c) {
+                            tmem_ld32(t_o + c * 32, o);
+                            tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t pk[16];
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const float2 x = fma2(make_float2(s[c * 32 + 2 * i], s[c * 32 + 2 * i + 1]), sc2, nm2);
-                            const float2 e = ((i % kPolyEvery) == kPolyEvery - 1)
-                                                 ? exp2_poly2(x)
-                                                 : make_float2(fast_exp2(x.x), fast_exp2(x.y));
-                            ps2 = add2(ps2, e);
-                            pk[i] = pack_bf16(e.x, e.y);
+                            for (int i = 0; i < 32; ++i) o[i] *= alpha;
+                            tmem_st32(t_o + c * 32, o);
                         }
-                        tmem_st16(t_s + c * 16, pk);
                     }
                 }
-                const float psum = ps2.x + ps2.y;
                 l_run += psum;
                 tmem_wait_st();
                 tc_fence_before();
