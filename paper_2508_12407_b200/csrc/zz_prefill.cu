@@ -35,7 +35,7 @@ constexpr int kTileBytes = 2 * kSubBytes;   // a full [128][128] bf16 tile
 constexpr int kStages = 4;                  // ring of K and V tiles (K_0, V_0, K_1, V_1, ...)
 constexpr int kThreads = 384;                // three warpgroups: softmax tile 0, softmax tile 1, TMA + MMA
 constexpr int kWarpTma = 8, kWarpMma = 9;
-constexpr int kRegsSoftmax = 224, kRegsAux = 56;   // 224 * 256 + 56 * 128 <= 65536 registers
+constexpr int kRegsSoftmax = 208, kRegsAux = 88;   // 208 * 256 + 88 * 128 <= 65536 registers
 constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 1024;
 constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr uint32_t kAbortPolls = 1u << 10;
@@ -157,6 +157,25 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_
         "mov.b64 db, {%2, %3};\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"((uint32_t)acc)
+        : "memory");
+}
+// Predicated forms (exec == 0: the instruction is issued but has no effect).  The thread that
+// issues the MMAs must not branch between them: the tensor pipe holds next to no queue, so every
+// cycle that thread spends resolving a branch is a cycle the pipe idles.
+__device__ __forceinline__ void mma_ss_if(uint32_t exec, uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t a_hi,
+                                          uint32_t b_hi, uint32_t idesc, bool acc) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\tsetp.ne.b32 q, %7, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"((uint32_t)acc), "r"(exec)
+        : "memory");
+}
+__device__ __forceinline__ void mma_commit_if(uint32_t exec, uint64_t* bar) {
+    asm volatile(
+        "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(smem_u32(bar)), "r"(exec)
         : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
@@ -436,55 +455,47 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
             for (int j = 0; j < n_tiles; ++j) {
                 const int uv = 2 * j + 1, uk = 2 * j + 2;
                 const int sv = uv % kStages, sk = uk % kStages;
-                const bool more = (j + 1) < n_tiles;
+                const uint32_t more = (j + 1) < n_tiles;
                 const uint32_t dvj = dv_lo + sv * kTile16, dkj = dk_lo + sk * kTile16;
+                // barriers of the next iteration (valid addresses and parities even past the end)
+                const int uv2 = uv + 2, uk2 = uk + 2;
+                uint64_t* next_v = &sh.kv_full[uv2 % kStages];
+                uint64_t* next_k = &sh.kv_full[uk2 % kStages];
+                const uint32_t next_v_par = (uv2 / kStages) & 1, next_k_par = (uk2 / kStages) & 1;
                 if (!ok_v) mbar_wait(&sh.kv_full[sv], (uv / kStages) & 1, &sh, p.status);
                 if (!ok_k) mbar_wait(&sh.kv_full[sk], (uk / kStages) & 1, &sh, p.status);
-                for (int t = 0; t < n_act; ++t) {
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (t == 1 && !active1) break;
                     if (!ok_p) mbar_wait(&sh.p_full[t], j & 1, &sh, p.status);
                     tc_fence_after();
                     const uint32_t t_st = tmem + t * 256;
                     const uint32_t dqt = dq_lo + t * kTile16;
-                    const bool last_of_iter = (t == n_act - 1);
-                    // probes for what is issued after this tile's MMAs
-                    auto probe_next = [&]() {
-                        if (!last_of_iter) {
-                            ok_p = mbar_test(&sh.p_full[1], j & 1);
-                        } else if (more) {
-                            const int uv2 = uv + 2, uk2 = uk + 2;
-                            ok_v = mbar_test(&sh.kv_full[uv2 % kStages], (uv2 / kStages) & 1);
-                            ok_k = (j + 2 < n_tiles) ? mbar_test(&sh.kv_full[uk2 % kStages], (uk2 / kStages) & 1) : true;
-                            ok_p = mbar_test(&sh.p_full[0], (j + 1) & 1);
-                        }
-                    };
+                    const uint32_t last_of_iter = (t == 1) ? 1u : (active1 ? 0u : 1u);
                     // O_t (+)= P_t V_j
-                    if (j > 0) {
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            if (kk == 6 && !more) probe_next();
-                            mma_ts(t_st + 128, t_st + kk * 8, dvj + kk * (2048 >> 4), dv_hi, kIdescPV, true);
-                        }
-                    } else {
+                    for (int kk = 0; kk < 8; ++kk)
+                        mma_ts(t_st + 128, t_st + kk * 8, dvj + kk * (2048 >> 4), dv_hi, kIdescPV, (kk > 0) || (j > 0));
+                    mma_commit_if(last_of_iter, &sh.kv_empty[sv]);
+                    // S_t = Q_t K_{j+1}^T (not after the last tile)
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            if (kk == 6 && !more) probe_next();
-                            mma_ts(t_st + 128, t_st + kk * 8, dvj + kk * (2048 >> 4), dv_hi, kIdescPV, kk > 0);
+                    for (int kk = 0; kk < 8; ++kk) {
+                        if (kk == 6) {
+                            // non-blocking probes of what is issued next; their latency hides behind the
+                            // last two MMAs
+                            if (t == 0 && active1) {
+                                ok_p = mbar_test(&sh.p_full[1], j & 1);
+                            } else {
+                                ok_v = mbar_test(next_v, next_v_par);
+                                ok_k = (j + 2 < n_tiles) ? mbar_test(next_k, next_k_par) : true;
+                                ok_p = mbar_test(&sh.p_full[0], (j + 1) & 1);
+                            }
                         }
+                        const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
+                        mma_ss_if(more, t_st, dqt + off16, dkj + off16, dkm_hi, dkm_hi, kIdescQK, kk > 0);
                     }
-                    if (last_of_iter) mma_commit(&sh.kv_empty[sv]);
-                    if (more) {
-                        // S_t = Q_t K_{j+1}^T
-#pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            if (kk == 6) probe_next();
-                            const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
-                            mma_ss(t_st, dqt + off16, dkj + off16, dkm_hi, dkm_hi, kIdescQK, kk > 0);
-                        }
-                    }
-                    if (more) {
-                        mma_commit(&sh.s_full[t]);
-                        if (last_of_iter) mma_commit(&sh.kv_empty[sk]);
-                    }
+                    mma_commit_if(more, &sh.s_full[t]);
+                    mma_commit_if(more & last_of_iter, &sh.kv_empty[sk]);
                 }
             }
             mma_commit(&sh.o_full);
