@@ -128,6 +128,7 @@ struct zz_cache {
     int num_sms;
     int decode_min_chunk;
     int decode_short_tokens;
+    int decode_overlap;
     bool has_mixed;
     alignas(64) CUtensorMap tmap_arena;
     bool have_tmap_arena;
@@ -263,7 +264,7 @@ void plan_splits(const zz_cache* c, const int* n, int Hg, int* warps, int* chunk
 // k_new/v_new != nullptr: fused append of one token per sequence (host lengths not yet bumped)
 int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q, __nv_bfloat16* out,
                         int q_head0, cudaStream_t st, const __nv_bfloat16* k_new = nullptr,
-                        const __nv_bfloat16* v_new = nullptr, int bump_len = 0) {
+                        const __nv_bfloat16* v_new = nullptr, int bump_len = 0, int overlap = 0) {
     const int Hg = (kind == ZZ_KIND_RETRIEVAL) ? c->nR[layer] : c->Hkv - c->nR[layer];
     if (Hg == 0) return ZZ_OK;
     zz::DecodeParams p;
@@ -306,7 +307,7 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
     const int items = p.split_start[c->B] * Hg;
     const int pk = (kind == ZZ_KIND_RETRIEVAL) ? zz::kProfDecodeR : zz::kProfDecodeS;
     zz::prof_begin(pk, st);
-    const cudaError_t e = zz::launch_decode(p, items, warps, st);
+    const cudaError_t e = zz::launch_decode(p, items, warps, st, overlap);
     zz::prof_end(pk, st);
     return e == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
 }
@@ -419,6 +420,7 @@ int zz_cache_create(const zz_config_t* cfg, void* d_arena, size_t arena_bytes, v
     c->max_new = cfg->max_new_tokens; c->scale = cfg->softmax_scale;
     c->decode_min_chunk = 256;
     c->decode_short_tokens = 384;
+    c->decode_overlap = 1;
     compute_layout(cfg, &c->lay, &c->desc);
     if (arena_bytes < c->lay.arena_bytes || workspace_bytes < c->lay.work_bytes) {
         delete c;
@@ -501,6 +503,10 @@ int zz_tune(zz_cache_t* c, const char* key, int value) {
         c->decode_min_chunk = value;
         return ZZ_OK;
     }
+    if (!strcmp(key, "decode_overlap")) {
+        c->decode_overlap = value != 0;
+        return ZZ_OK;
+    }
     if (!strcmp(key, "decode_short_tokens")) {
         if (value < 0 || value % 16) return ZZ_ERR_INVALID_ARG;
         c->decode_short_tokens = value;
@@ -574,8 +580,18 @@ int zz_decode_attn(zz_cache_t* c, int layer, const void* d_q, void* d_out, void*
     return r;
 }
 
+static int decode_step_impl(zz_cache_t* c, int layer, const void* d_q, const void* d_k, const void* d_v,
+                            void* d_out, void* stream, int overlap);
+
 int zz_decode_step(zz_cache_t* c, int layer, const void* d_q, const void* d_k, const void* d_v, void* d_out,
                    void* stream) {
+    return decode_step_impl(c, layer, d_q, d_k, d_v, d_out, stream, 0);
+}
+
+// overlap: the launch may start while the previous launch in the stream drains (exclusive layers
+// only; the caller guarantees that launch belonged to another layer and did not produce q/k/v)
+static int decode_step_impl(zz_cache_t* c, int layer, const void* d_q, const void* d_k, const void* d_v,
+                            void* d_out, void* stream, int overlap) {
     if (bad_layer(c, layer) || !d_q || !d_k || !d_v || !d_out) return ZZ_ERR_INVALID_ARG;
     if (((uintptr_t)d_q | (uintptr_t)d_k | (uintptr_t)d_v | (uintptr_t)d_out) & 15) return ZZ_ERR_INVALID_ARG;
     const int nR = c->nR[layer];
@@ -593,7 +609,7 @@ int zz_decode_step(zz_cache_t* c, int layer, const void* d_q, const void* d_k, c
     int r;
     if (!c->mixed(layer)) {
         const int kind = nR ? ZZ_KIND_RETRIEVAL : ZZ_KIND_STREAMING;
-        r = launch_decode_group(c, layer, kind, q, out, 0, st, k, v, 1);
+        r = launch_decode_group(c, layer, kind, q, out, 0, st, k, v, 1, overlap && c->decode_overlap);
     } else {
         r = regroup(c, layer, q, c->d_qc(), c->B, 1, st);
         if (r == ZZ_OK) r = launch_decode_group(c, layer, ZZ_KIND_RETRIEVAL, c->d_qc(), c->d_oc(), 0, st, k, v, 0);
@@ -615,10 +631,12 @@ int zz_decode_step_all(zz_cache_t* c, const void* d_q, const void* d_k, const vo
         for (int b = 0; b < c->B; ++b)
             if (c->nR[l] > 0 && c->len[(size_t)l * c->B + b] + 1 > c->cap[b]) return ZZ_ERR_CAPACITY;
     for (int l = 0; l < c->L; ++l) {
-        const int r = zz_decode_step(c, l, static_cast<const char*>(d_q) + l * qs,
-                                     static_cast<const char*>(d_k) + l * ks,
-                                     static_cast<const char*>(d_v) + l * ks,
-                                     static_cast<char*>(d_out) + l * qs, stream);
+        // q/k/v of every layer are inputs of this call, and layer l's launch reads nothing that layer
+        // l-1's launches write before its griddepcontrol.wait, so consecutive layers may overlap
+        const int r = decode_step_impl(c, l, static_cast<const char*>(d_q) + l * qs,
+                                       static_cast<const char*>(d_k) + l * ks,
+                                       static_cast<const char*>(d_v) + l * ks,
+                                       static_cast<char*>(d_out) + l * qs, stream, l > 0);
         if (r != ZZ_OK) return r;
     }
     return ZZ_OK;

@@ -102,7 +102,7 @@ struct PrefillParams {
 
 // ---- launchers (defined in the .cu files) -------------------------------------------
 cudaError_t launch_append(const AppendParams& p, int grid_x, cudaStream_t s);
-cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStream_t s);
+cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStream_t s, int overlap = 0);
 cudaError_t launch_regroup(const GatherParams& p, cudaStream_t s);
 cudaError_t launch_reset(int* len, int* pos, int L, int B, int ring, int seq, cudaStream_t s);
 cudaError_t decode_setup();

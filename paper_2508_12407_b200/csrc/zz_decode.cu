@@ -14,6 +14,8 @@
 // the split merge, so there is no second launch.
 //
 // The roofline of this kernel is HBM bandwidth: 2 * 128 * 2 bytes per token and KV head.
+#include <cstring>
+
 #include "zz_common.cuh"
 
 namespace zz {
@@ -105,6 +107,12 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int grp = lane >> 2, tig = lane & 3;
+
+    // Programmatic dependent launch (no-ops in an ordinary launch): the next launch in the stream
+    // may start as soon as every CTA of this one is running, and fills the SMs this launch leaves
+    // idle in its tail; this launch in turn touches what the previous one may still be using (the
+    // shared split workspace, the counters, the output) only after griddepcontrol.wait below.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---- which work item -----------------------------------------------------------
     const int item = blockIdx.x;
@@ -270,6 +278,8 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
         __syncwarp();
     }
     cp_async_wait<0>();
+    // everything up to here read only this layer's stores, lengths and the caller's q/k/v
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- merge the warps of this CTA ---------------------------------------------------------
 #pragma unroll
@@ -429,21 +439,32 @@ cudaError_t decode_setup() {
     return e;
 }
 
-cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStream_t s) {
+// overlap != 0: programmatic stream serialization -- the launch may begin while the previous launch
+// in the stream is still draining.  Only for launches whose early reads (this layer's stores and
+// lengths, the caller's q/k/v) the previous launch cannot have written.
+cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStream_t s, int overlap) {
     if (n_items <= 0) return cudaSuccess;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(n_items);
+    cfg.blockDim = dim3(warps == 8 ? 256 : 128);
+    cfg.dynamicSmemBytes = (warps == 8 ? 8 : 4) * kWarpSmem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    cudaError_t e;
     if (warps == 8) {
-        if (p.G > 8)
-            decode_kernel<true, 8><<<n_items, 256, 8 * kWarpSmem, s>>>(p);
-        else
-            decode_kernel<false, 8><<<n_items, 256, 8 * kWarpSmem, s>>>(p);
+        if (p.G > 8) e = cudaLaunchKernelEx(&cfg, decode_kernel<true, 8>, p);
+        else e = cudaLaunchKernelEx(&cfg, decode_kernel<false, 8>, p);
     } else {
-        if (p.G > 8)
-            decode_kernel<true, 4><<<n_items, 128, 4 * kWarpSmem, s>>>(p);
-        else
-            decode_kernel<false, 4><<<n_items, 128, 4 * kWarpSmem, s>>>(p);
+        if (p.G > 8) e = cudaLaunchKernelEx(&cfg, decode_kernel<true, 4>, p);
+        else e = cudaLaunchKernelEx(&cfg, decode_kernel<false, 4>, p);
     }
     count_launch();
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace zz
