@@ -55,6 +55,7 @@ using zz::SeqDesc;
 namespace {
 
 constexpr int kMaxSplits = 120;   // the decode kernel keeps per-split factors in 128-entry rows
+constexpr int kMaxSlots = 512;    // upper bound of CTAs a long-store decode plan may use (2 per SM)
 constexpr size_t kAlign = 256;
 
 size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
@@ -63,7 +64,7 @@ struct Layout {
     // workspace sections (byte offsets)
     size_t off_status, off_len, off_pos, off_desc, off_heads, off_counters, off_part_ml, off_part_o,
         off_qc, off_oc, work_bytes;
-    size_t arena_bytes;
+    size_t arena_bytes, counters_per_layer, items_per_layer;
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -139,9 +140,15 @@ struct zz_cache {
     int* d_pos(int l) const { return reinterpret_cast<int*>(work + lay.off_pos) + (size_t)l * B * ring; }
     SeqDesc* d_desc(int l) const { return reinterpret_cast<SeqDesc*>(work + lay.off_desc) + (size_t)l * B; }
     int* d_heads(int l) const { return reinterpret_cast<int*>(work + lay.off_heads) + (size_t)l * Hkv; }
-    unsigned int* d_counters() const { return reinterpret_cast<unsigned int*>(work + lay.off_counters); }
-    float* d_part_ml() const { return reinterpret_cast<float*>(work + lay.off_part_ml); }
-    float* d_part_o() const { return reinterpret_cast<float*>(work + lay.off_part_o); }
+    unsigned int* d_counters(int l) const {
+        return reinterpret_cast<unsigned int*>(work + lay.off_counters) + (size_t)l * lay.counters_per_layer;
+    }
+    float* d_part_ml(int l) const {
+        return reinterpret_cast<float*>(work + lay.off_part_ml) + (size_t)l * lay.items_per_layer * G * 2;
+    }
+    float* d_part_o(int l) const {
+        return reinterpret_cast<float*>(work + lay.off_part_o) + (size_t)l * lay.items_per_layer * G * kD;
+    }
     __nv_bfloat16* d_qc() const { return reinterpret_cast<__nv_bfloat16*>(work + lay.off_qc); }
     __nv_bfloat16* d_oc() const { return reinterpret_cast<__nv_bfloat16*>(work + lay.off_oc); }
     __nv_bfloat16* d_arena() const { return reinterpret_cast<__nv_bfloat16*>(arena); }
@@ -208,9 +215,14 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
     lay->off_pos = w; w += align_up((size_t)L * B * ring * sizeof(int));
     lay->off_desc = w; w += align_up((size_t)L * B * sizeof(SeqDesc));
     lay->off_heads = w; w += align_up((size_t)L * Hkv * sizeof(int));
-    lay->off_counters = w; w += align_up((size_t)(B * Hkv + B) * sizeof(unsigned int));
-    lay->off_part_ml = w; w += align_up((size_t)B * Hkv * kMaxSplits * G * 2 * sizeof(float));
-    lay->off_part_o = w; w += align_up((size_t)B * Hkv * kMaxSplits * G * kD * sizeof(float));
+    // per layer: arrival counters and the split partials of the layer's launches, indexed by work
+    // item (at most kMaxSlots + B * Hkv items per launch), so that the launches of different
+    // layers share no scratch and may overlap
+    lay->counters_per_layer = (size_t)(B * Hkv + B);
+    lay->items_per_layer = (size_t)kMaxSlots + (size_t)B * Hkv;
+    lay->off_counters = w; w += align_up((size_t)L * lay->counters_per_layer * sizeof(unsigned int));
+    lay->off_part_ml = w; w += align_up((size_t)L * lay->items_per_layer * G * 2 * sizeof(float));
+    lay->off_part_o = w; w += align_up((size_t)L * lay->items_per_layer * G * kD * sizeof(float));
     lay->off_qc = w;
     if (has_mixed) w += align_up((size_t)c->max_new_tokens * Hq * kD * 2);
     lay->off_oc = w;
@@ -238,7 +250,7 @@ void plan_splits(const zz_cache* c, const int* n, int Hg, int* warps, int* chunk
         return;
     }
     *warps = 4;
-    const int slots = 2 * c->num_sms;
+    const int slots = 2 * c->num_sms < kMaxSlots ? 2 * c->num_sms : kMaxSlots;
     long long per = (total * Hg + slots - 1) / slots;   // tokens per work item if all were equal
     if (per < c->decode_min_chunk) per = c->decode_min_chunk;
     for (;;) {
@@ -276,7 +288,7 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
     p.v_new = v_new;
     p.head_list = c->d_heads(layer);
     p.pos = c->d_pos(layer);
-    p.seq_counters = c->d_counters() + (size_t)c->B * c->Hkv;
+    p.seq_counters = c->d_counters(layer) + (size_t)c->B * c->Hkv;
     p.kv_head0 = (kind == ZZ_KIND_RETRIEVAL) ? 0 : c->nR[layer];
     p.n_kv_total = c->Hkv;
     p.S = c->S;
@@ -286,9 +298,9 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
     p.out = out;
     p.q_tok_stride = (long long)c->Hq * kD;
     p.q_head0 = q_head0;
-    p.part_o = c->d_part_o();
-    p.part_ml = c->d_part_ml();
-    p.counters = c->d_counters();
+    p.part_o = c->d_part_o(layer);
+    p.part_ml = c->d_part_ml(layer);
+    p.counters = c->d_counters(layer);
     p.status = c->d_status();
     p.kind = kind;
     p.ring = c->ring;
@@ -420,7 +432,7 @@ int zz_cache_create(const zz_config_t* cfg, void* d_arena, size_t arena_bytes, v
     c->max_new = cfg->max_new_tokens; c->scale = cfg->softmax_scale;
     c->decode_min_chunk = 256;
     c->decode_short_tokens = 384;
-    c->decode_overlap = 1;
+    c->decode_overlap = 2;
     compute_layout(cfg, &c->lay, &c->desc);
     if (arena_bytes < c->lay.arena_bytes || workspace_bytes < c->lay.work_bytes) {
         delete c;
@@ -504,7 +516,8 @@ int zz_tune(zz_cache_t* c, const char* key, int value) {
         return ZZ_OK;
     }
     if (!strcmp(key, "decode_overlap")) {
-        c->decode_overlap = value != 0;
+        if (value < 0 || value > 2) return ZZ_ERR_INVALID_ARG;
+        c->decode_overlap = value;
         return ZZ_OK;
     }
     if (!strcmp(key, "decode_short_tokens")) {
@@ -609,7 +622,7 @@ static int decode_step_impl(zz_cache_t* c, int layer, const void* d_q, const voi
     int r;
     if (!c->mixed(layer)) {
         const int kind = nR ? ZZ_KIND_RETRIEVAL : ZZ_KIND_STREAMING;
-        r = launch_decode_group(c, layer, kind, q, out, 0, st, k, v, 1, overlap && c->decode_overlap);
+        r = launch_decode_group(c, layer, kind, q, out, 0, st, k, v, 1, overlap ? c->decode_overlap : 0);
     } else {
         r = regroup(c, layer, q, c->d_qc(), c->B, 1, st);
         if (r == ZZ_OK) r = launch_decode_group(c, layer, ZZ_KIND_RETRIEVAL, c->d_qc(), c->d_oc(), 0, st, k, v, 0);

@@ -44,8 +44,8 @@ struct DecodeParams {
     __nv_bfloat16* out;      // same addressing as q
     long long q_tok_stride;  // elements between consecutive sequences' rows (n_q_heads * 128)
     int q_head0;             // first query head of this group inside a row
-    float* part_o;           // [B*Hg][max_splits][G][128]
-    float* part_ml;          // [B*Hg][max_splits][G][2]
+    float* part_o;           // [work item][G][128] split partials of this launch
+    float* part_ml;          // [work item][G][2]
     unsigned int* counters;  // [B*Hg], 0 between launches
     int* status;
     int kind;                // which group of the layer
@@ -64,6 +64,7 @@ struct DecodeParams {
     int n_kv_total;
     int S, W;
     int bump_len;            // this launch advances len (the last launch of a layer does)
+    int gdc_wait;            // wait for the previous launch before touching workspace and output
     int split_start[ZZ_MAX_BATCH + 1];  // prefix sum of per-sequence split counts
     int chunk[ZZ_MAX_BATCH];            // tokens per split of each sequence
     SeqDesc sd[ZZ_MAX_BATCH];           // store addresses of every sequence of this layer

@@ -110,8 +110,9 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
 
     // Programmatic dependent launch (no-ops in an ordinary launch): the next launch in the stream
     // may start as soon as every CTA of this one is running, and fills the SMs this launch leaves
-    // idle in its tail; this launch in turn touches what the previous one may still be using (the
-    // shared split workspace, the counters, the output) only after griddepcontrol.wait below.
+    // idle in its tail.  A launch that shares anything with its predecessor (gdc_wait) touches it
+    // only after griddepcontrol.wait below; the layers of one decode step share nothing (own
+    // stores, lengths, split workspace and output slice) and run without that wait.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---- which work item -----------------------------------------------------------
@@ -279,7 +280,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     }
     cp_async_wait<0>();
     // everything up to here read only this layer's stores, lengths and the caller's q/k/v
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (p.gdc_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- merge the warps of this CTA ---------------------------------------------------------
 #pragma unroll
@@ -307,10 +308,10 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     }
     __syncthreads();
 
-    const int d = threadIdx.x & 127;   // 128 output dims; with 8 warps the halves split the rows
     const long long pair = (long long)b * p.Hg + hg;
     __nv_bfloat16* outb = p.out + ((long long)b * p.q_tok_stride) + (long long)(p.q_head0 + hg * G) * kD;
-    for (int row = threadIdx.x >> 7; row < G; row += kWarps / 4) {
+    for (int idx = threadIdx.x; idx < G * kD; idx += kWarps * 32) {
+        const int row = idx >> 7, d = idx & 127;
         float M = -INFINITY;
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) M = fmaxf(M, sm_ml[(w * 16 + row) * 2]);
@@ -325,7 +326,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
         if (nsplit == 1) {
             outb[row * kD + d] = __float2bfloat16_rn(acc / L);
         } else {
-            const long long po = ((pair * p.max_splits + split) * G + row);
+            const long long po = (long long)item * G + row;   // partials are indexed by work item
             p.part_o[po * kD + d] = acc;
             if (d == 0) {
                 p.part_ml[po * 2 + 0] = M;
@@ -367,8 +368,10 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     for (int row0 = 0; row0 < G; row0 += kWarps) {
         const int row = row0 + warp;                         // this warp's row (4 dims per lane)
         const bool row_ok = row < G;
-        const float* pbase = p.part_o + ((pair * p.max_splits) * G + (row_ok ? row : 0)) * kD + lane * 4;
-        const long long sstride = (long long)G * kD;
+        // split s of this (sequence, head) is work item item0 + s * Hg
+        const long long item0 = (long long)p.split_start[b] * p.Hg + hg;
+        const float* pbase = p.part_o + (item0 * G + (row_ok ? row : 0)) * kD + lane * 4;
+        const long long sstride = (long long)p.Hg * G * kD;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int sb = 0; sb < nsplit; sb += kRound) {
             float4 v[kRound];
@@ -380,7 +383,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
                 for (int i = threadIdx.x; i < nsplit * kWarps; i += blockDim.x) {
                     const int s = i / kWarps, r = row0 + i % kWarps;
                     if (r < G) {
-                        const long long po = ((pair * p.max_splits + s) * G + r);
+                        const long long po = (item0 + (long long)s * p.Hg) * G + r;
                         const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + po * 2));
                         sm_m[r * kMaxSplitsSmem + s] = ml.x;
                         sm_f[r * kMaxSplitsSmem + s] = ml.y;
@@ -436,32 +439,42 @@ cudaError_t decode_setup() {
         e = cudaFuncSetAttribute(decode_kernel<false, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * kWarpSmem);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(decode_kernel<true, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * kWarpSmem);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(decode_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kWarpSmem);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(decode_kernel<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kWarpSmem);
     return e;
 }
 
 // overlap != 0: programmatic stream serialization -- the launch may begin while the previous launch
 // in the stream is still draining.  Only for launches whose early reads (this layer's stores and
-// lengths, the caller's q/k/v) the previous launch cannot have written.
+// lengths, the caller's q/k/v) the previous launch cannot have written.  overlap == 2: the launch
+// shares nothing at all with the previous one and does not wait for it.
 cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStream_t s, int overlap) {
     if (n_items <= 0) return cudaSuccess;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(n_items);
-    cfg.blockDim = dim3(warps == 8 ? 256 : 128);
-    cfg.dynamicSmemBytes = (warps == 8 ? 8 : 4) * kWarpSmem;
+    cfg.blockDim = dim3(warps * 32);
+    cfg.dynamicSmemBytes = warps * kWarpSmem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
+    DecodeParams pp = p;
+    pp.gdc_wait = (overlap == 2) ? 0 : 1;
     cudaError_t e;
     if (warps == 8) {
-        if (p.G > 8) e = cudaLaunchKernelEx(&cfg, decode_kernel<true, 8>, p);
-        else e = cudaLaunchKernelEx(&cfg, decode_kernel<false, 8>, p);
+        if (p.G > 8) e = cudaLaunchKernelEx(&cfg, decode_kernel<true, 8>, pp);
+        else e = cudaLaunchKernelEx(&cfg, decode_kernel<false, 8>, pp);
+    } else if (warps == 2) {
+        if (p.G > 8) e = cudaLaunchKernelEx(&cfg, decode_kernel<true, 2>, pp);
+        else e = cudaLaunchKernelEx(&cfg, decode_kernel<false, 2>, pp);
     } else {
-        if (p.G > 8) e = cudaLaunchKernelEx(&cfg, decode_kernel<true, 4>, p);
-        else e = cudaLaunchKernelEx(&cfg, decode_kernel<false, 4>, p);
+        if (p.G > 8) e = cudaLaunchKernelEx(&cfg, decode_kernel<true, 4>, pp);
+        else e = cudaLaunchKernelEx(&cfg, decode_kernel<false, 4>, pp);
     }
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();

@@ -131,6 +131,54 @@ def test_min_chunk_tuning_keeps_results():
         assert_close(got, want, "tuned split")
 
 
+def test_whole_stack_step_overlap_modes_agree():
+    """zz_decode_step_all with its layers overlapped (programmatic dependent launch, with and
+    without the wait between layers) gives the same bits as plain stream order, and matches the
+    oracle: the layers of a step share no scratch."""
+    import torch
+    D, L, B, Hq, Hkv, S, W = 128, 6, 2, 8, 2, 16, 48
+    kinds = [1, 0, 1, 1, 0, 1]
+    lens = [5000, 2300]
+    steps = 12
+    w = inputs.Workload("t", L, B, Hq, Hkv, D, S, W, 4, 0, 0, steps, seed=4242)
+    hist = [[inputs.qkv_bf16(w, l, b, 0, lens[b]) for b in range(B)] for l in range(L)]
+    dec = [[[inputs.qkv_bf16(w, l, b, lens[b] + i, 1) for b in range(B)] for l in range(L)] for i in range(steps)]
+    results = {}
+    for mode in (0, 1, 2):
+        cache = make(L, B, Hq, Hkv, S, W, kinds, [n + steps + 4 for n in lens], max_new=8192)
+        cache.tune("decode_overlap", mode)
+        for l in range(L):
+            k = np.concatenate([hist[l][b][1] for b in range(B)])
+            v = np.concatenate([hist[l][b][2] for b in range(B)])
+            cache.kv_append(l, to_dev(k), to_dev(v), lens)
+        outs = []
+        for i in range(steps):
+            q = np.stack([np.concatenate([dec[i][l][b][0] for b in range(B)]) for l in range(L)])
+            k = np.stack([np.concatenate([dec[i][l][b][1] for b in range(B)]) for l in range(L)])
+            v = np.stack([np.concatenate([dec[i][l][b][2] for b in range(B)]) for l in range(L)])
+            dq, dk, dv = to_dev(q), to_dev(k), to_dev(v)
+            out = torch.zeros_like(dq)
+            cache.decode_step_all(dq, dk, dv, out)
+            outs.append(to_bits(out))
+        torch.cuda.synchronize()
+        assert cache.last_status() == 0
+        results[mode] = np.stack(outs)
+        cache.close()
+    assert np.array_equal(results[0], results[1]) and np.array_equal(results[0], results[2])
+    # last step of every layer and sequence against the oracle
+    scale = 1 / np.sqrt(D)
+    for l in range(L):
+        for b in range(B):
+            o = OracleSeq(Hkv, D, S, W, lens[b] + steps + 4, [kinds[l]] * Hkv)
+            o.append(hist[l][b][1], hist[l][b][2])
+            for i in range(steps):
+                o.append(dec[i][l][b][1], dec[i][l][b][2])
+            t = lens[b] + steps - 1
+            want = o.rows(dec[steps - 1][l][b][0], [t], scale=scale)
+            got = results[2][steps - 1, l, b:b + 1]
+            assert_close(got, want, f"layer {l} seq {b}")
+
+
 def test_error_paths_leave_cache_untouched():
     cache = make(2, 1, 8, 2, 4, 8, [1, 0], [10])
     w = inputs.Workload("t", 2, 1, 8, 2, 128, 4, 8, 1, 0, 0, 1, seed=3)
