@@ -158,6 +158,11 @@ size_t zz_stage_bytes(const zz_cache_t* cache, int64_t n_tokens);
 int zz_decode_step_host(zz_cache_t* cache, int layer, const void* h_q, const void* h_k,
                         const void* h_v, void* h_out, void* d_stage, size_t stage_bytes,
                         void* stream);
+/* zz_decode_step_all fed from HOST memory: h_q/h_out [n_layers, batch, n_q_heads, 128], h_k/h_v
+ * [n_layers, batch, n_kv_heads, 128]; d_stage holds at least
+ * zz_stage_bytes(cache, n_layers * batch) bytes. */
+int zz_decode_step_all_host(zz_cache_t* cache, const void* h_q, const void* h_k, const void* h_v,
+                            void* h_out, void* d_stage, size_t stage_bytes, void* stream);
 int zz_prefill_host(zz_cache_t* cache, int layer, const void* h_q, const void* h_k,
                     const void* h_v, void* h_out, const int32_t* h_n_new, void* d_stage,
                     size_t stage_bytes, void* stream);

@@ -75,6 +75,7 @@ SYMBOLS = {
     "zz_profile_read": (_i32, [_i32, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double), _i32]),
     "zz_stage_bytes": (_sz, [_vp, _i64]),
     "zz_decode_step_host": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "zz_decode_step_all_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "zz_prefill_host": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "zz_cache_export_shape": (_i32, [_vp, _i32, _i32, _i32, ctypes.POINTER(ctypes.c_int32),
                                      ctypes.POINTER(ctypes.c_int32)]),
@@ -264,6 +265,11 @@ class ZigzagCache:
         _check(self._lib.zz_decode_step_host(self._h, layer, _dptr(h_q), _dptr(h_k), _dptr(h_v),
                                              _dptr(h_out), _dptr(d_stage), d_stage.numel(),
                                              _stream_ptr(stream)), "zz_decode_step_host")
+
+    def decode_step_all_host(self, h_q, h_k, h_v, h_out, d_stage, stream=None) -> None:
+        _check(self._lib.zz_decode_step_all_host(self._h, _dptr(h_q), _dptr(h_k), _dptr(h_v), _dptr(h_out),
+                                                 _dptr(d_stage), d_stage.numel(), _stream_ptr(stream)),
+               "zz_decode_step_all_host")
 
     def prefill_host(self, layer: int, h_q, h_k, h_v, h_out, n_new, d_stage, stream=None) -> None:
         nn = self._n_new(n_new)

@@ -765,6 +765,26 @@ int zz_decode_step_host(zz_cache_t* c, int layer, const void* h_q, const void* h
     return run_host(c, layer, h_q, h_k, h_v, h_out, ones, d_stage, stage_bytes, stream, true);
 }
 
+int zz_decode_step_all_host(zz_cache_t* c, const void* h_q, const void* h_k, const void* h_v, void* h_out,
+                            void* d_stage, size_t stage_bytes, void* stream) {
+    if (!c || !h_q || !h_k || !h_v || !h_out || !d_stage) return ZZ_ERR_INVALID_ARG;
+    const long long total = (long long)c->L * c->B;
+    if (stage_bytes < zz_stage_bytes(c, total)) return ZZ_ERR_WORKSPACE;
+    if ((uintptr_t)d_stage % kAlign) return ZZ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t qbytes = (size_t)total * c->Hq * kD * 2, kbytes = (size_t)total * c->Hkv * kD * 2;
+    const size_t qb = align_up(qbytes), kb = align_up(kbytes);
+    unsigned char* s = static_cast<unsigned char*>(d_stage);
+    void* dq = s; void* dk = s + qb; void* dv = s + qb + kb; void* dout = s + qb + 2 * kb;
+    if (cudaMemcpyAsync(dq, h_q, qbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    if (cudaMemcpyAsync(dk, h_k, kbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    if (cudaMemcpyAsync(dv, h_v, kbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    const int r = zz_decode_step_all(c, dq, dk, dv, dout, stream);
+    if (r != ZZ_OK) return r;
+    if (cudaMemcpyAsync(h_out, dout, qbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    return ZZ_OK;
+}
+
 int zz_prefill_host(zz_cache_t* c, int layer, const void* h_q, const void* h_k, const void* h_v, void* h_out,
                     const int32_t* h_n_new, void* d_stage, size_t stage_bytes, void* stream) {
     return run_host(c, layer, h_q, h_k, h_v, h_out, h_n_new, d_stage, stage_bytes, stream, false);
