@@ -190,6 +190,9 @@ def run_ours(args, w):
     cache = binding.ZigzagCache(L, B, Hq, Hkv, w.sink, w.recent, kinds, cap, max(B, B * C), kvhead_is_retrieval=kvk,
                                 device=f"cuda:{local}")
 
+    if args.decode_overlap >= 0:
+        cache.tune("decode_overlap", args.decode_overlap)
+
     gen = torch.Generator(device=dev)
     gen.manual_seed(w.seed + 1000 * rank)
 
@@ -370,7 +373,7 @@ def run_ours(args, w):
             "config": {"workload": w.name + ("+mixed" if args.mixed else ""), "layers": L, "batch": B,
                        "q_heads": Hq, "kv_heads": Hkv, "head_dim": D, "sink": w.sink, "recent": w.recent,
                        "retrieval_layers": nR_layers, "prefill_len": w.prefill_len, "prefill_chunk": C,
-                       "decode_steps": steps_dec,
+                       "decode_steps": steps_dec, "decode_overlap": args.decode_overlap if args.decode_overlap >= 0 else 2,
                        "context": [int(x) for x in lens] if not C else w.prefill_len,
                        "l2": "per-layer inputs larger than L2 (KV per retrieval layer %.0f MB)" % (
                            2 * Hkv * float(base_len.mean()) * D * 2 / 1e6),
@@ -444,6 +447,8 @@ def main():
     ap.add_argument("--share-inputs", action="store_true", help="one set of prefill tensors for all layers")
     ap.add_argument("--profile-period", type=int, default=8,
                     help="bracket every n-th launch of each kernel class with CUDA events (0 = off)")
+    ap.add_argument("--decode-overlap", type=int, default=-1, choices=[-1, 0, 1, 2],
+                    help="override how the decode launches of consecutive layers follow one another (library default: 2)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -228,6 +228,22 @@ int zz_decode_attn_static(const void* d_q, const void* d_k, const void* d_v, voi
 int zz_decode_attn_static_limits(int32_t* max_batch, int32_t* max_batch_times_q_heads,
                                  size_t* scratch_bytes);
 
+/* Layer-mask solver (paper: Section 2.2 "Transport Optimization", Eq. 5; the quantile split it
+ * starts from is the last paragraph of Section 2.1).  Host function, no device work.
+ *   h_alpha [n_layers * n_heads]  per-head importances (the converged alpha of the head-importance
+ *                                 training; larger = needs full attention), finite
+ *   n_streaming_layers = p        layers that become all-streaming; the quantile split marks the
+ *                                 p * n_heads heads of smallest alpha as streaming heads (sparsity p / L)
+ *   omega in [0, 1]               weight of the gain of turning a streaming head into a retrieval head
+ * Writes h_layer_is_retrieval [n_layers] (1 = retrieval layer): the choice of p streaming layers
+ * that minimises Eq. 5's sum over heads of  alpha (retrieval head made streaming), -omega * alpha
+ * (streaming head made retrieval), 0 (kept).  Equal costs: the lower layer index becomes streaming.
+ * Optional outputs (may be NULL): h_head_is_retrieval [n_layers * n_heads], the quantile split;
+ * *h_cost, the minimum.  Returns ZZ_ERR_INVALID_ARG on NULL / out-of-range / non-finite input. */
+int zz_layer_mask_solve(const float* h_alpha, int32_t n_layers, int32_t n_heads, int32_t n_streaming_layers,
+                        double omega, uint8_t* h_layer_is_retrieval, uint8_t* h_head_is_retrieval,
+                        double* h_cost);
+
 /* Number of kernels this library has launched since it was loaded (all handles). */
 int64_t zz_launch_count(void);
 

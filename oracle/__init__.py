@@ -53,6 +53,10 @@ def _load() -> ctypes.CDLL:
     lib.zzo_attn_from_slots.argtypes = [vp, i64, vp, vp, vp, i64, i32, i32, i32, vp, i64, i64, dbl, vp]
     lib.zzo_attn_from_slots.restype = i32
     lib.zzo_num_threads.restype = i32
+    lib.zzo_layer_mask_enumerate.argtypes = [vp, vp, i32, i32, i32, dbl, vp, vp, vp]
+    lib.zzo_layer_mask_enumerate.restype = i32
+    lib.zzo_quantile_split.argtypes = [vp, i32, i32, vp]
+    lib.zzo_quantile_split.restype = i32
     _lib = lib
     return lib
 
@@ -125,6 +129,32 @@ def attn_from_slots(q: np.ndarray, t: int, store_k: np.ndarray, store_v: np.ndar
     if rc != 0:
         raise ValueError(f"zzo_attn_from_slots failed: {rc}")
     return out
+
+
+def quantile_split(alpha: np.ndarray, n_streaming: int) -> np.ndarray:
+    """uint8 mask over the flattened heads: 0 for the n_streaming heads of smallest alpha."""
+    a = np.ascontiguousarray(alpha, dtype=np.float64).ravel()
+    out = np.zeros(a.size, dtype=np.uint8)
+    rc = _load().zzo_quantile_split(_ptr(a), a.size, int(n_streaming), _ptr(out))
+    if rc != 0:
+        raise ValueError(f"zzo_quantile_split failed: {rc}")
+    return out.reshape(np.shape(alpha))
+
+
+def layer_mask_enumerate(alpha: np.ndarray, head_is_retr: np.ndarray, p: int, omega: float):
+    """Exhaustive minimisation of Eq. 5 over all subsets of p streaming layers.
+    Returns (layer_is_retrieval uint8 [L], minimum cost, second smallest cost)."""
+    a = np.ascontiguousarray(alpha, dtype=np.float64)
+    L, H = a.shape
+    hr = np.ascontiguousarray(head_is_retr, dtype=np.uint8)
+    assert hr.shape == (L, H)
+    out = np.zeros(L, dtype=np.uint8)
+    best, second = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    rc = _load().zzo_layer_mask_enumerate(_ptr(a), _ptr(hr), L, H, int(p), float(omega), _ptr(out),
+                                          ctypes.byref(best), ctypes.byref(second))
+    if rc != 0:
+        raise ValueError(f"zzo_layer_mask_enumerate failed: {rc}")
+    return out, float(best.value), float(second.value)
 
 
 class RingStore:

@@ -37,6 +37,9 @@
  * v_t; |V(t)| = min(t+1, S+W); decode step t == prefill row t; chunked == single
  * shot; ring route == full-history route; occupied ring positions; invariance
  * under slot permutation; GQA replication; mixed layer == per-head kinds.
+ * Layer-mask choice (Eq. 5, at the end of this file): a hand-worked example (tests/golden),
+ * the same objective written per layer in numpy over itertools subsets, the already-exclusive
+ * split costing nothing, omega = 0 reducing to the least retrieval mass, head-order invariance.
  */
 #include <math.h>
 #include <stdint.h>
@@ -242,4 +245,64 @@ int zzo_num_threads(void) {
 #else
     return 1;
 #endif
+}
+
+/*
+ * Layer-mask choice by exhaustive enumeration (Section 2.2, Eq. 5), as the paper describes it:
+ * every subset of p streaming layers is examined one by one and the one of minimum cost kept.
+ *   alpha            [L][H]  head importances
+ *   head_is_retr     [L][H]  the quantile split the transition starts from (1 = retrieval head)
+ *   p                        number of all-streaming layers
+ *   omega                    scaling factor of the third case
+ *   best_is_retr     [L]     out: 1 = retrieval layer, for the first subset (in increasing binary
+ *                            order of the streaming-layer bit mask) that attains the minimum
+ *   best_cost, second_cost   out: the minimum and the smallest cost of any other subset
+ * Per head (i, j), with the layer's new kind k_i:  0 if the head keeps its kind;  alpha_ij if a
+ * retrieval head becomes a streaming head;  -omega * alpha_ij if a streaming head becomes a
+ * retrieval head.  L <= 24.
+ */
+int zzo_layer_mask_enumerate(const double* alpha, const uint8_t* head_is_retr, int L, int H, int p,
+                             double omega, uint8_t* best_is_retr, double* best_cost, double* second_cost) {
+    if (!alpha || !head_is_retr || !best_is_retr || !best_cost || !second_cost) return ZZO_BAD_ARG;
+    if (L < 1 || L > 24 || H < 1 || p < 0 || p > L) return ZZO_BAD_ARG;
+    double best = INFINITY, second = INFINITY;
+    uint32_t best_mask = 0;
+    for (uint32_t mask = 0; mask < (1u << L); ++mask) {          /* bit i set: layer i becomes streaming */
+        int bits = 0;
+        for (int i = 0; i < L; ++i) bits += (mask >> i) & 1u;
+        if (bits != p) continue;
+        double cost = 0.0;
+        for (int i = 0; i < L; ++i) {
+            const int layer_streaming = (mask >> i) & 1u;
+            for (int j = 0; j < H; ++j) {
+                const int was_retr = head_is_retr[i * H + j] ? 1 : 0;
+                double hat;
+                if (was_retr && layer_streaming) hat = alpha[i * H + j];                 /* o(1) */
+                else if (!was_retr && !layer_streaming) hat = -omega * alpha[i * H + j]; /* o(2) */
+                else hat = 0.0;                                                          /* o(0) */
+                cost += hat;
+            }
+        }
+        if (cost < best) { second = best; best = cost; best_mask = mask; }
+        else if (cost < second) second = cost;
+    }
+    for (int i = 0; i < L; ++i) best_is_retr[i] = ((best_mask >> i) & 1u) ? 0 : 1;
+    *best_cost = best;
+    *second_cost = second;
+    return ZZO_OK;
+}
+
+/* Quantile split (Section 2.1, last paragraph): the n_streaming heads of smallest alpha become
+ * streaming heads; among equal alphas the earlier (layer, head) first.  Selection by repeated
+ * minimum search, no sort. */
+int zzo_quantile_split(const double* alpha, int n, int n_streaming, uint8_t* is_retr) {
+    if (!alpha || !is_retr || n < 1 || n_streaming < 0 || n_streaming > n) return ZZO_BAD_ARG;
+    for (int i = 0; i < n; ++i) is_retr[i] = 1;
+    for (int r = 0; r < n_streaming; ++r) {
+        int arg = -1;
+        for (int i = 0; i < n; ++i)
+            if (is_retr[i] && (arg < 0 || alpha[i] < alpha[arg])) arg = i;
+        is_retr[arg] = 0;
+    }
+    return ZZO_OK;
 }

@@ -82,6 +82,7 @@ SYMBOLS = {
     "zz_cache_export": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, ctypes.POINTER(ctypes.c_int32), _vp]),
     "zz_cache_import": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp]),
     "zz_get_last_status": (_i32, [_vp, _vp]),
+    "zz_layer_mask_solve": (_i32, [_vp, _i32, _i32, _i32, ctypes.c_double, _vp, _vp, ctypes.POINTER(ctypes.c_double)]),
     "zz_decode_attn_static": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, ctypes.c_float, _vp]),
     "zz_decode_attn_static_limits": (_i32, [ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
                                             ctypes.POINTER(_sz)]),
@@ -329,6 +330,19 @@ def decode_attn_static_limits():
     _check(load().zz_decode_attn_static_limits(ctypes.byref(mb), ctypes.byref(mr), ctypes.byref(sb)),
            "zz_decode_attn_static_limits")
     return int(mb.value), int(mr.value), int(sb.value)
+
+
+def layer_mask_solve(alpha: np.ndarray, n_streaming_layers: int, omega: float):
+    """Layer-mask solver (Eq. 5): alpha [n_layers, n_heads] -> (layer_is_retrieval uint8 [n_layers],
+    head_is_retrieval uint8 [n_layers, n_heads] of the quantile split, minimum cost)."""
+    a = np.ascontiguousarray(alpha, dtype=np.float32)
+    L, H = a.shape
+    layers = np.zeros(L, dtype=np.uint8)
+    heads = np.zeros((L, H), dtype=np.uint8)
+    cost = ctypes.c_double(0.0)
+    _check(load().zz_layer_mask_solve(_np_ptr(a), L, H, int(n_streaming_layers), float(omega), _np_ptr(layers),
+                                      _np_ptr(heads), ctypes.byref(cost)), "zz_layer_mask_solve")
+    return layers, heads, float(cost.value)
 
 
 def bf16_bits_to_tensor(bits: np.ndarray, device="cuda:0"):
