@@ -668,24 +668,39 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
             mbar_wait(&sh.o_full, 0, &sh, p.status);
             tc_fence_after();
             const float inv = 1.f / l_run;
-            const bool row_ok = rr < C;
-            __nv_bfloat16* orow = p.out + (long long)(p.tok_off[b] + rr) * p.tok_stride +
-                                  (long long)(p.q_head0 + hg * p.G + g0 + t) * kD;
+            // Every MMA of this CTA has completed, so the tile's Q buffer is free: the warp stages its
+            // 32 rows there (16-byte pieces XOR-swizzled by row) and writes them out with every
+            // 256-byte row covered by 16 consecutive lanes, instead of one lane per row.
+            const uint32_t stage = sm_q + t * kTileBytes + (uint32_t)(quarter * 32) * 256;
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
                 float o[32];
                 tmem_ld32(t_o + c * 32, o);
                 tmem_wait_ld();
-                if (row_ok) {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        uint4 w;
-                        w.x = pack_bf16(o[8 * i + 0] * inv, o[8 * i + 1] * inv);
-                        w.y = pack_bf16(o[8 * i + 2] * inv, o[8 * i + 3] * inv);
-                        w.z = pack_bf16(o[8 * i + 4] * inv, o[8 * i + 5] * inv);
-                        w.w = pack_bf16(o[8 * i + 6] * inv, o[8 * i + 7] * inv);
-                        *reinterpret_cast<uint4*>(orow + c * 32 + i * 8) = w;
-                    }
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t w0 = pack_bf16(o[8 * i + 0] * inv, o[8 * i + 1] * inv);
+                    const uint32_t w1 = pack_bf16(o[8 * i + 2] * inv, o[8 * i + 3] * inv);
+                    const uint32_t w2 = pack_bf16(o[8 * i + 4] * inv, o[8 * i + 5] * inv);
+                    const uint32_t w3 = pack_bf16(o[8 * i + 6] * inv, o[8 * i + 7] * inv);
+                    const uint32_t piece = (uint32_t)(c * 4 + i);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + lane * 256 + ((piece ^ (lane & 15)) << 4)),
+                                 "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+                }
+            }
+            __syncwarp();
+            {
+                const int piece = lane & 15, half = lane >> 4;
+                const long long row0 = (long long)p.tok_off[b] + r0 + quarter * 32;
+                __nv_bfloat16* obase = p.out + (long long)(p.q_head0 + hg * p.G + g0 + t) * kD + piece * 8;
+#pragma unroll 4
+                for (int i = 0; i < 16; ++i) {
+                    const int lr = 2 * i + half;                           // row inside the warp's 32
+                    uint32_t w0, w1, w2, w3;
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
+                                 : "r"(stage + lr * 256 + ((piece ^ (lr & 15)) << 4)) : "memory");
+                    if (r0 + quarter * 32 + lr < C)
+                        *reinterpret_cast<uint4*>(obase + (row0 + lr) * p.tok_stride) = make_uint4(w0, w1, w2, w3);
                 }
             }
         }
