@@ -130,6 +130,7 @@ struct zz_cache {
     int decode_min_chunk;
     int decode_short_tokens;
     int decode_overlap;
+    bool last_nowait;   // the last launch did not wait for its predecessor: the next one must be an ordinary launch
     bool has_mixed;
     alignas(64) CUtensorMap tmap_arena;
     bool have_tmap_arena;
@@ -319,6 +320,11 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
     const int items = p.split_start[c->B] * Hg;
     const int pk = (kind == ZZ_KIND_RETRIEVAL) ? zz::kProfDecodeR : zz::kProfDecodeS;
     zz::prof_begin(pk, st);
+    // A programmatic launch orders itself only against its immediate predecessor.  After a launch
+    // that did not wait for its own predecessor, only an ordinary launch (full stream order) or
+    // another launch of the same independent chain may follow.
+    if (c->last_nowait && overlap != 2) overlap = 0;
+    c->last_nowait = (overlap == 2);
     const cudaError_t e = zz::launch_decode(p, items, warps, st, overlap);
     zz::prof_end(pk, st);
     return e == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
@@ -335,7 +341,8 @@ int regroup(zz_cache* c, int layer, const __nv_bfloat16* src, __nv_bfloat16* dst
     g.tokens = tokens;
     g.to_compact = to_compact;
     zz::prof_begin(zz::kProfRegroup, st);
-    const cudaError_t e = zz::launch_regroup(g, st);
+    const cudaError_t e = zz::launch_regroup(g, st, c->last_nowait ? 0 : 1);
+    c->last_nowait = false;
     zz::prof_end(zz::kProfRegroup, st);
     return e == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
 }
@@ -382,6 +389,7 @@ int launch_prefill_group(zz_cache* c, int layer, int kind, const CUtensorMap* tq
     if (items > 0x7fffffffLL) return ZZ_ERR_UNSUPPORTED;
     const int pk = (kind == ZZ_KIND_RETRIEVAL) ? zz::kProfPrefillR : zz::kProfPrefillS;
     zz::prof_begin(pk, st);
+    c->last_nowait = false;   // an ordinary launch: full stream order
     const cudaError_t e = zz::launch_prefill(p, tq, tk, tv, &c->tmap_arena, (int)items, st);
     zz::prof_end(pk, st);
     return e == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
@@ -433,6 +441,7 @@ int zz_cache_create(const zz_config_t* cfg, void* d_arena, size_t arena_bytes, v
     c->decode_min_chunk = 256;
     c->decode_short_tokens = 384;
     c->decode_overlap = 2;
+    c->last_nowait = false;
     compute_layout(cfg, &c->lay, &c->desc);
     if (arena_bytes < c->lay.arena_bytes || workspace_bytes < c->lay.work_bytes) {
         delete c;
@@ -494,6 +503,7 @@ int zz_cache_destroy(zz_cache_t* c) {
 int zz_cache_reset(zz_cache_t* c, int seq, void* stream) {
     if (!c || seq < -1 || seq >= c->B) return ZZ_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    c->last_nowait = false;
     if (zz::launch_reset(c->d_len(0), c->d_pos(0), c->L, c->B, c->ring, seq, st) != cudaSuccess)
         return ZZ_ERR_CUDA;
     for (int l = 0; l < c->L; ++l)
@@ -565,6 +575,7 @@ int zz_kv_append(zz_cache_t* c, int layer, const void* d_k, const void* d_v, con
     const long long gx = (worst + 255) / 256;
     if (gx > 0x7fffffffLL) return ZZ_ERR_UNSUPPORTED;
     zz::prof_begin(zz::kProfAppend, static_cast<cudaStream_t>(stream));
+    c->last_nowait = false;
     const cudaError_t ae = zz::launch_append(p, (int)gx, static_cast<cudaStream_t>(stream));
     zz::prof_end(zz::kProfAppend, static_cast<cudaStream_t>(stream));
     if (ae != cudaSuccess) return ZZ_ERR_CUDA;
@@ -582,13 +593,15 @@ int zz_decode_attn(zz_cache_t* c, int layer, const void* d_q, void* d_out, void*
     __nv_bfloat16* out = static_cast<__nv_bfloat16*>(d_out);
     if (!c->mixed(layer)) {
         const int kind = c->nR[layer] ? ZZ_KIND_RETRIEVAL : ZZ_KIND_STREAMING;
-        return launch_decode_group(c, layer, kind, q, out, 0, st);
+        return launch_decode_group(c, layer, kind, q, out, 0, st, nullptr, nullptr, 0, c->decode_overlap ? 3 : 0);
     }
     // DuoAttention-style layer: gather the heads of each kind, one pass per kind, scatter back
     int r = regroup(c, layer, q, c->d_qc(), c->B, 1, st);
-    if (r == ZZ_OK) r = launch_decode_group(c, layer, ZZ_KIND_RETRIEVAL, c->d_qc(), c->d_oc(), 0, st);
+    const int ov = c->decode_overlap ? 3 : 0;
+    if (r == ZZ_OK) r = launch_decode_group(c, layer, ZZ_KIND_RETRIEVAL, c->d_qc(), c->d_oc(), 0, st, nullptr, nullptr, 0, ov);
     if (r == ZZ_OK)
-        r = launch_decode_group(c, layer, ZZ_KIND_STREAMING, c->d_qc(), c->d_oc(), c->nR[layer] * c->G, st);
+        r = launch_decode_group(c, layer, ZZ_KIND_STREAMING, c->d_qc(), c->d_oc(), c->nR[layer] * c->G, st, nullptr,
+                                nullptr, 0, ov);
     if (r == ZZ_OK) r = regroup(c, layer, c->d_oc(), out, c->B, 0, st);
     return r;
 }
@@ -622,12 +635,13 @@ static int decode_step_impl(zz_cache_t* c, int layer, const void* d_q, const voi
     int r;
     if (!c->mixed(layer)) {
         const int kind = nR ? ZZ_KIND_RETRIEVAL : ZZ_KIND_STREAMING;
-        r = launch_decode_group(c, layer, kind, q, out, 0, st, k, v, 1, overlap ? c->decode_overlap : 0);
+        r = launch_decode_group(c, layer, kind, q, out, 0, st, k, v, 1, overlap ? c->decode_overlap : (c->decode_overlap ? 3 : 0));
     } else {
         r = regroup(c, layer, q, c->d_qc(), c->B, 1, st);
-        if (r == ZZ_OK) r = launch_decode_group(c, layer, ZZ_KIND_RETRIEVAL, c->d_qc(), c->d_oc(), 0, st, k, v, 0);
+        const int ov = c->decode_overlap ? 3 : 0;
+        if (r == ZZ_OK) r = launch_decode_group(c, layer, ZZ_KIND_RETRIEVAL, c->d_qc(), c->d_oc(), 0, st, k, v, 0, ov);
         if (r == ZZ_OK)
-            r = launch_decode_group(c, layer, ZZ_KIND_STREAMING, c->d_qc(), c->d_oc(), nR * c->G, st, k, v, 1);
+            r = launch_decode_group(c, layer, ZZ_KIND_STREAMING, c->d_qc(), c->d_oc(), nR * c->G, st, k, v, 1, ov);
         if (r == ZZ_OK) r = regroup(c, layer, c->d_oc(), out, c->B, 0, st);
     }
     if (r != ZZ_OK) return r;

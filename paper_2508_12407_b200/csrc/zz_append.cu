@@ -1,5 +1,7 @@
 // KV append with sink + recent eviction, cache reset, and the head regrouping copies of the
 // mixed-head layer.  All three are pure data movement: 16-byte vector loads and stores.
+#include <cstring>
+
 #include "zz_common.cuh"
 
 namespace zz {
@@ -101,6 +103,10 @@ cudaError_t launch_reset(int* len, int* pos, int L, int B, int ring, int seq, cu
 // [token][Hkv*G][128] and the compact group order (retrieval heads first, then streaming),
 // 16 bytes per thread.
 __global__ void __launch_bounds__(256) regroup_kernel(const GatherParams p) {
+    // launched with programmatic stream serialization: the launch itself overlaps the previous
+    // kernel's tail, the data dependence is kept by waiting here before anything is read
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const long long total = p.tokens * p.Hkv * p.G * 16;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
@@ -120,14 +126,24 @@ __global__ void __launch_bounds__(256) regroup_kernel(const GatherParams p) {
     }
 }
 
-cudaError_t launch_regroup(const GatherParams& p, cudaStream_t s) {
+cudaError_t launch_regroup(const GatherParams& p, cudaStream_t s, int programmatic) {
     const long long total = p.tokens * p.Hkv * p.G * 16;
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
     if (blocks < 1) blocks = 1;
-    regroup_kernel<<<(int)blocks, 256, 0, s>>>(p);
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(256);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = programmatic ? 1 : 0;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, regroup_kernel, p);
     count_launch();
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace zz

@@ -64,7 +64,8 @@ struct DecodeParams {
     int n_kv_total;
     int S, W;
     int bump_len;            // this launch advances len (the last launch of a layer does)
-    int gdc_wait;            // wait for the previous launch before touching workspace and output
+    int gdc_wait;            // 1: wait for the previous launch before touching workspace and output;
+                             // 2: wait at kernel entry; 0: never
     int split_start[ZZ_MAX_BATCH + 1];  // prefix sum of per-sequence split counts
     int chunk[ZZ_MAX_BATCH];            // tokens per split of each sequence
     SeqDesc sd[ZZ_MAX_BATCH];           // store addresses of every sequence of this layer
@@ -104,7 +105,7 @@ struct PrefillParams {
 // ---- launchers (defined in the .cu files) -------------------------------------------
 cudaError_t launch_append(const AppendParams& p, int grid_x, cudaStream_t s);
 cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStream_t s, int overlap = 0);
-cudaError_t launch_regroup(const GatherParams& p, cudaStream_t s);
+cudaError_t launch_regroup(const GatherParams& p, cudaStream_t s, int programmatic);
 cudaError_t launch_reset(int* len, int* pos, int L, int B, int ring, int seq, cudaStream_t s);
 cudaError_t decode_setup();
 cudaError_t prefill_setup();

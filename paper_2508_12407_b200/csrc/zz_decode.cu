@@ -113,6 +113,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     // idle in its tail.  A launch that shares anything with its predecessor (gdc_wait) touches it
     // only after griddepcontrol.wait below; the layers of one decode step share nothing (own
     // stores, lengths, split workspace and output slice) and run without that wait.
+    if (p.gdc_wait == 2) asm volatile("griddepcontrol.wait;" ::: "memory");   // before anything is read
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---- which work item -----------------------------------------------------------
@@ -449,7 +450,9 @@ cudaError_t decode_setup() {
 // overlap != 0: programmatic stream serialization -- the launch may begin while the previous launch
 // in the stream is still draining.  Only for launches whose early reads (this layer's stores and
 // lengths, the caller's q/k/v) the previous launch cannot have written.  overlap == 2: the launch
-// shares nothing at all with the previous one and does not wait for it.
+// shares nothing at all with the previous one and does not wait for it.  overlap == 3: the kernel
+// waits for the previous launch at entry, before it reads anything (always safe; only the launch
+// latency overlaps).
 cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStream_t s, int overlap) {
     if (n_items <= 0) return cudaSuccess;
     cudaLaunchConfig_t cfg;
@@ -464,7 +467,7 @@ cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStr
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
     DecodeParams pp = p;
-    pp.gdc_wait = (overlap == 2) ? 0 : 1;
+    pp.gdc_wait = (overlap == 2) ? 0 : (overlap == 3) ? 2 : 1;
     cudaError_t e;
     if (warps == 8) {
         if (p.G > 8) e = cudaLaunchKernelEx(&cfg, decode_kernel<true, 8>, pp);
