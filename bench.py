@@ -159,7 +159,7 @@ def run_reference(args, w):
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
-    from paper_2508_12407_b200 import binding, build
+    from paper_2508_12407_b200 import binding, build, replicas
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -194,7 +194,7 @@ def run_ours(args, w):
         cache.tune("decode_overlap", args.decode_overlap)
 
     gen = torch.Generator(device=dev)
-    gen.manual_seed(w.seed + 1000 * rank)
+    gen.manual_seed(replicas.replica_seed(w.seed, rank))
 
     def randn(*shape):
         return torch.randn(*shape, device=dev, generator=gen, dtype=torch.float32).to(torch.bfloat16)
@@ -273,14 +273,10 @@ def run_ours(args, w):
     total_ms = t0.elapsed_time(t1)
     pre_ms = sum(m[0].elapsed_time(m[1]) for m in all_marks)
     dec_ms = sum(m[1].elapsed_time(m[2]) for m in all_marks)
-    tms = torch.tensor([total_ms, pre_ms, dec_ms], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-    total_ms, pre_ms, dec_ms = (float(x) for x in tms.tolist())
+    total_ms, pre_ms, dec_ms = replicas.max_over_ranks([total_ms, pre_ms, dec_ms], dev)
 
     K = args.steps
-    tokens_dec = world * B * steps_dec * K
-    us_per_token = dec_ms * 1e3 / tokens_dec if tokens_dec else float("nan")
+    us_per_token = replicas.whole_job_us_per_token(dec_ms, world, B, steps_dec * K)
 
     # ---- algorithmic work -----------------------------------------------------------------
     nR_layers = int(kinds.sum()) if kvk is None else None
