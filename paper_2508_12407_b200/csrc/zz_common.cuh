@@ -96,6 +96,7 @@ struct PrefillParams {
     int n_kv_total;          // KV heads per row of the chunk K/V
     int ring, S, W, Hg, G, B;
     int total_tiles;         // 128-row query tiles over the whole batch
+    int n_items;             // work items of the launch (set by the launcher)
     float scale_log2;
     int n_new[ZZ_MAX_BATCH];
     int tok_off[ZZ_MAX_BATCH];

@@ -36,7 +36,8 @@ constexpr int kStages = 4;                  // ring of K and V tiles (K_0, V_0, 
 constexpr int kThreads = 384;                // three warpgroups: softmax tile 0, softmax tile 1, TMA + MMA
 constexpr int kWarpTma = 8, kWarpMma = 9;
 constexpr int kRegsSoftmax = 208, kRegsAux = 88;   // 208 * 256 + 88 * 128 <= 65536 registers
-constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 1024;
+constexpr int kEpiBytes = 8 * 4096;          // output staging: 16 rows of 256 B per softmax warp
+constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + kEpiBytes + 1024;
 constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr uint32_t kAbortPolls = 1u << 10;
 constexpr float kRescaleThreshold = 8.f;    // log2 units of slack before O is rescaled
@@ -51,6 +52,7 @@ constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);   // B (= V) is MN-major
 
 struct Shared {
     uint64_t q_full;
+    uint64_t q_empty;          // the item's last Q K^T has completed: the Q buffer may be reloaded
     uint64_t kv_full[kStages];
     uint64_t kv_empty[kStages];
     uint64_t s_full[2];
@@ -325,6 +327,47 @@ __device__ __forceinline__ void plan_tile(const TilePlan& t, int j, bool& is_chu
     }
 }
 
+// One work item = (128-token query tile, KV head of the group, pair of query heads).  A CTA is
+// persistent: it works through items k = 0, 1, ... of a static boustrophedon schedule over the
+// items in long-first order (wave w forwards, wave w+1 backwards), so every CTA gets nearly the same
+// number of KV tiles, the TMA producer runs ahead into the next item, and tensor-memory allocation,
+// barrier set-up and the first loads are paid once per CTA instead of once per item.
+struct Item {
+    int b, qt, r0, C, P, hg, g0, n_tiles;
+    bool active1;
+    TilePlan plan;
+};
+__device__ __forceinline__ int item_index(int k, int n_items) {
+    const int g = (int)gridDim.x;
+    const int idx = k * g + ((k & 1) ? g - 1 - (int)blockIdx.x : (int)blockIdx.x);
+    return idx < n_items ? idx : -1;
+}
+__device__ __forceinline__ Item get_item(const PrefillParams& p, int idx) {
+    Item it;
+    const int pairs = (p.G + 1) >> 1;
+    const int per_tile = p.Hg * pairs;
+    const int ti = idx / per_tile;
+    const int rem = idx % per_tile;
+    it.hg = rem / pairs;
+    it.g0 = (rem % pairs) * 2;
+    it.active1 = (it.g0 + 1) < p.G;
+    const int gt = p.total_tiles - 1 - ti;      // long (late) tiles first
+    int b = 0;
+    while (b + 1 < p.B && gt >= p.tile_start[b + 1]) ++b;
+    it.b = b;
+    it.qt = gt - p.tile_start[b];
+    it.r0 = it.qt * kTile;
+    it.C = p.n_new[b];
+    it.P = p.len[b];
+    it.plan = make_plan(p.kind, it.P, it.C, it.qt, p.S, p.W, p.ring);
+    it.n_tiles = it.plan.n_total;
+    return it;
+}
+
+// kPersistent = false: one item per CTA (grid = items); the item loops below then run once and
+// every running counter folds to a constant.  Long retrieval items gain nothing from persistence
+// and run a few per cent faster this way; the short items of streaming layers gain ~10 %.
+template <bool kPersistent>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q,
                const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
@@ -337,26 +380,12 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    // ---- work item: (query tile, KV head of the group, pair of query heads) ---------------------
-    const int pairs = (p.G + 1) >> 1;
-    const int per_tile = p.Hg * pairs;
-    const int it = blockIdx.x / per_tile;
-    const int rem = blockIdx.x % per_tile;
-    const int hg = rem / pairs;
-    const int g0 = (rem % pairs) * 2;
-    const bool active1 = (g0 + 1) < p.G;
-    const int gt = p.total_tiles - 1 - it;      // long (late) tiles first
-    int b = 0;
-    while (b + 1 < p.B && gt >= p.tile_start[b + 1]) ++b;
-    const int qt = gt - p.tile_start[b];
-    const int r0 = qt * kTile;
-    const int C = p.n_new[b];
-    const int P = p.len[b];
-    const TilePlan plan = make_plan(p.kind, P, C, qt, p.S, p.W, p.ring);
-    const int n_tiles = plan.n_total;
+    const int n_items = p.n_items;
+    const uint32_t sm_epi = smem_base + 2 * kTileBytes + kStages * kTileBytes;   // output staging
 
     if (threadIdx.x == 0) {
         mbar_init(&sh.q_full, 1);
+        mbar_init(&sh.q_empty, 1);
         for (int i = 0; i < kStages; ++i) {
             mbar_init(&sh.kv_full[i], 1);
             mbar_init(&sh.kv_empty[i], 1);
@@ -386,139 +415,169 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
       if (warp == kWarpTma) {
         // ================= TMA producer =================
         if (lane == 0) {
-            const SeqDesc sd = p.desc[b];
-            const long long slots_per_head = (p.kind == ZZ_KIND_RETRIEVAL) ? sd.cap : p.ring;
-            const int k_row0 = (int)(sd.k_off[p.kind] / kD + (long long)hg * slots_per_head);
-            const int v_row0 = (int)(sd.v_off[p.kind] / kD + (long long)hg * slots_per_head);
-            const int src_head = p.head_list[p.kv_head0 + hg];
-            const int tok0 = p.tok_off[b];
-            const int qh = p.q_head0 + hg * p.G + g0;
-            mbar_expect_tx(&sh.q_full, active1 ? 2 * kTileBytes : kTileBytes);
-            tma_load_3d(sm_q, &tmap_q, 0, qh, tok0 + r0, &sh.q_full);
-            tma_load_3d(sm_q + kSubBytes, &tmap_q, 64, qh, tok0 + r0, &sh.q_full);
-            if (active1) {
-                tma_load_3d(sm_q + kTileBytes, &tmap_q, 0, qh + 1, tok0 + r0, &sh.q_full);
-                tma_load_3d(sm_q + kTileBytes + kSubBytes, &tmap_q, 64, qh + 1, tok0 + r0, &sh.q_full);
-            }
-            for (int u = 0; u < 2 * n_tiles; ++u) {
-                const int stage = u % kStages;
-                mbar_wait(&sh.kv_empty[stage], ((u / kStages) & 1) ^ 1, &sh, p.status);
-                bool is_chunk;
-                int start;
-                plan_tile(plan, u >> 1, is_chunk, start);
-                const bool is_v = u & 1;
-                const uint32_t dst = sm_kv + stage * kTileBytes;
-                mbar_expect_tx(&sh.kv_full[stage], kTileBytes);
-                if (is_chunk) {
-                    const CUtensorMap* m = is_v ? &tmap_v : &tmap_k;
-                    tma_load_3d(dst, m, 0, src_head, tok0 + start, &sh.kv_full[stage]);
-                    tma_load_3d(dst + kSubBytes, m, 64, src_head, tok0 + start, &sh.kv_full[stage]);
-                } else {
-                    const int row = (is_v ? v_row0 : k_row0) + start;
-                    tma_load_2d(dst, &tmap_arena, 0, row, &sh.kv_full[stage]);
-                    tma_load_2d(dst + kSubBytes, &tmap_arena, 64, row, &sh.kv_full[stage]);
+            uint32_t u_glob = 0;                      // K/V sub-tiles loaded so far (all items)
+            for (int k = 0;; ++k) {
+                if (!kPersistent && k > 0) break;
+                const int idx = kPersistent ? item_index(k, n_items) : (int)blockIdx.x;
+                if (idx < 0) break;
+                const Item it = get_item(p, idx);
+                const SeqDesc sd = p.desc[it.b];
+                const long long slots_per_head = (p.kind == ZZ_KIND_RETRIEVAL) ? sd.cap : p.ring;
+                const int k_row0 = (int)(sd.k_off[p.kind] / kD + (long long)it.hg * slots_per_head);
+                const int v_row0 = (int)(sd.v_off[p.kind] / kD + (long long)it.hg * slots_per_head);
+                const int src_head = p.head_list[p.kv_head0 + it.hg];
+                const int tok0 = p.tok_off[it.b];
+                const int qh = p.q_head0 + it.hg * p.G + it.g0;
+                if (k > 0) mbar_wait(&sh.q_empty, (k - 1) & 1, &sh, p.status);
+                mbar_expect_tx(&sh.q_full, it.active1 ? 2 * kTileBytes : kTileBytes);
+                tma_load_3d(sm_q, &tmap_q, 0, qh, tok0 + it.r0, &sh.q_full);
+                tma_load_3d(sm_q + kSubBytes, &tmap_q, 64, qh, tok0 + it.r0, &sh.q_full);
+                if (it.active1) {
+                    tma_load_3d(sm_q + kTileBytes, &tmap_q, 0, qh + 1, tok0 + it.r0, &sh.q_full);
+                    tma_load_3d(sm_q + kTileBytes + kSubBytes, &tmap_q, 64, qh + 1, tok0 + it.r0, &sh.q_full);
+                }
+                for (int u = 0; u < 2 * it.n_tiles; ++u, ++u_glob) {
+                    const int stage = u_glob % kStages;
+                    mbar_wait(&sh.kv_empty[stage], ((u_glob / kStages) & 1) ^ 1, &sh, p.status);
+                    bool is_chunk;
+                    int start;
+                    plan_tile(it.plan, u >> 1, is_chunk, start);
+                    const bool is_v = u & 1;
+                    const uint32_t dst = sm_kv + stage * kTileBytes;
+                    mbar_expect_tx(&sh.kv_full[stage], kTileBytes);
+                    if (is_chunk) {
+                        const CUtensorMap* m = is_v ? &tmap_v : &tmap_k;
+                        tma_load_3d(dst, m, 0, src_head, tok0 + start, &sh.kv_full[stage]);
+                        tma_load_3d(dst + kSubBytes, m, 64, src_head, tok0 + start, &sh.kv_full[stage]);
+                    } else {
+                        const int row = (is_v ? v_row0 : k_row0) + start;
+                        tma_load_2d(dst, &tmap_arena, 0, row, &sh.kv_full[stage]);
+                        tma_load_2d(dst + kSubBytes, &tmap_arena, 64, row, &sh.kv_full[stage]);
+                    }
                 }
             }
         }
       } else if (warp == kWarpMma) {
         // ================= MMA issuer =================
         if (lane == 0) {
-            const int n_act = active1 ? 2 : 1;
             const uint64_t dq = make_desc(sm_q, 16, 1024);          // Q tile 0, K-major
             const uint64_t dk = make_desc(sm_kv, 16, 1024);         // K tile in stage 0, K-major
             const uint64_t dv = make_desc(sm_kv, kSubBytes, 1024);  // V tile in stage 0, MN-major
             const uint32_t dq_lo = (uint32_t)dq, dk_lo = (uint32_t)dk, dv_lo = (uint32_t)dv;
             const uint32_t dkm_hi = (uint32_t)(dq >> 32), dv_hi = (uint32_t)(dv >> 32);
             constexpr uint32_t kTile16 = kTileBytes >> 4;
-            mbar_wait(&sh.q_full, 0, &sh, p.status);
-            mbar_wait(&sh.kv_full[0], 0, &sh, p.status);
-            tc_fence_after();
-            // S_t = Q_t K_0^T
-            for (int t = 0; t < n_act; ++t) {
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
-                    mma_ss(tmem + t * 256, dq_lo + t * kTile16 + off16, dk_lo + off16, dkm_hi, dkm_hi, kIdescQK,
-                           kk > 0);
-                }
-                mma_commit(&sh.s_full[t]);
-            }
-            mma_commit(&sh.kv_empty[0]);
-            // The thread that issues tcgen05.mma is held at each one until the tensor pipe has room, so
-            // whatever it does between two tiles leaves the pipe idle.  The barriers of the next tile
-            // (K/V stages, the other tile's P) are therefore probed two MMAs before the current
-            // tile's last one; the probe's latency then overlaps those MMAs, and the blocking wait is
-            // only entered when a probe came back negative.
-            bool ok_v = mbar_test(&sh.kv_full[1 % kStages], 0);
-            bool ok_k = (n_tiles > 1) ? mbar_test(&sh.kv_full[2 % kStages], 0) : true;
-            bool ok_p = mbar_test(&sh.p_full[0], 0);
-            for (int j = 0; j < n_tiles; ++j) {
-                const int uv = 2 * j + 1, uk = 2 * j + 2;
-                const int sv = uv % kStages, sk = uk % kStages;
-                const uint32_t more = (j + 1) < n_tiles;
-                const uint32_t dvj = dv_lo + sv * kTile16, dkj = dk_lo + sk * kTile16;
-                // barriers of the next iteration (valid addresses and parities even past the end)
-                const int uv2 = uv + 2, uk2 = uk + 2;
-                uint64_t* next_v = &sh.kv_full[uv2 % kStages];
-                uint64_t* next_k = &sh.kv_full[uk2 % kStages];
-                const uint32_t next_v_par = (uv2 / kStages) & 1, next_k_par = (uk2 / kStages) & 1;
-                if (!ok_v) mbar_wait(&sh.kv_full[sv], (uv / kStages) & 1, &sh, p.status);
-                if (!ok_k) mbar_wait(&sh.kv_full[sk], (uk / kStages) & 1, &sh, p.status);
-#pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    if (t == 1 && !active1) break;
-                    if (!ok_p) mbar_wait(&sh.p_full[t], j & 1, &sh, p.status);
-                    tc_fence_after();
-                    const uint32_t t_st = tmem + t * 256;
-                    const uint32_t dqt = dq_lo + t * kTile16;
-                    const uint32_t last_of_iter = (t == 1) ? 1u : (active1 ? 0u : 1u);
-                    // O_t (+)= P_t V_j
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        mma_ts(t_st + 128, t_st + kk * 8, dvj + kk * (2048 >> 4), dv_hi, kIdescPV, (kk > 0) || (j > 0));
-                    mma_commit_if(last_of_iter, &sh.kv_empty[sv]);
-                    // S_t = Q_t K_{j+1}^T (not after the last tile)
+            // Counters that run across the items of this CTA (barrier phases never restart):
+            uint32_t u_glob = 0;          // K/V sub-tiles consumed
+            uint32_t ph[2] = {0, 0};      // S/P tiles handled per query tile (tile 1 only in items that have it)
+            for (int k = 0;; ++k) {
+                if (!kPersistent && k > 0) break;
+                const int idx = kPersistent ? item_index(k, n_items) : (int)blockIdx.x;
+                if (idx < 0) break;
+                const Item it = get_item(p, idx);
+                const int n_tiles = it.n_tiles;
+                const bool active1 = it.active1;
+                const int n_act = active1 ? 2 : 1;
+                mbar_wait(&sh.q_full, k & 1, &sh, p.status);
+                mbar_wait(&sh.kv_full[u_glob % kStages], (u_glob / kStages) & 1, &sh, p.status);
+                tc_fence_after();
+                // S_t = Q_t K_0^T
+                for (int t = 0; t < n_act; ++t) {
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
-                        if (kk == 6) {
-                            // non-blocking probes of what is issued next; their latency hides behind the
-                            // last two MMAs
-                            if (t == 0 && active1) {
-                                ok_p = mbar_test(&sh.p_full[1], j & 1);
-                            } else {
-                                ok_v = mbar_test(next_v, next_v_par);
-                                ok_k = (j + 2 < n_tiles) ? mbar_test(next_k, next_k_par) : true;
-                                ok_p = mbar_test(&sh.p_full[0], (j + 1) & 1);
-                            }
-                        }
                         const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
-                        mma_ss_if(more, t_st, dqt + off16, dkj + off16, dkm_hi, dkm_hi, kIdescQK, kk > 0);
+                        mma_ss(tmem + t * 256, dq_lo + t * kTile16 + off16,
+                               dk_lo + (u_glob % kStages) * kTile16 + off16, dkm_hi, dkm_hi, kIdescQK, kk > 0);
                     }
-                    mma_commit_if(more, &sh.s_full[t]);
-                    mma_commit_if(more & last_of_iter, &sh.kv_empty[sk]);
+                    mma_commit(&sh.s_full[t]);
                 }
+                mma_commit(&sh.kv_empty[u_glob % kStages]);
+                mma_commit_if(n_tiles == 1, &sh.q_empty);
+                // The thread that issues tcgen05.mma is held at each one until the tensor pipe has room,
+                // so whatever it does between two tiles leaves the pipe idle.  The barriers of the next
+                // tile (K/V stages, the other tile's P) are therefore probed, without blocking, two MMAs
+                // before the current tile's last one; the probe's latency then overlaps those MMAs, and
+                // the blocking wait is only entered when a probe came back negative.
+                bool ok_v = false, ok_k = false, ok_p = false;
+                for (int j = 0; j < n_tiles; ++j) {
+                    const uint32_t uv = u_glob + 2 * j + 1, uk = u_glob + 2 * j + 2;
+                    const uint32_t sv = uv % kStages, sk = uk % kStages;
+                    const uint32_t more = (j + 1) < n_tiles;
+                    const uint32_t dvj = dv_lo + sv * kTile16, dkj = dk_lo + sk * kTile16;
+                    // barriers of the next iteration (valid addresses and parities even past the end)
+                    const uint32_t uv2 = uv + 2, uk2 = uk + 2;
+                    uint64_t* next_v = &sh.kv_full[uv2 % kStages];
+                    uint64_t* next_k = &sh.kv_full[uk2 % kStages];
+                    const uint32_t next_v_par = (uv2 / kStages) & 1, next_k_par = (uk2 / kStages) & 1;
+                    if (!ok_v) mbar_wait(&sh.kv_full[sv], (uv / kStages) & 1, &sh, p.status);
+                    if (!ok_k && more) mbar_wait(&sh.kv_full[sk], (uk / kStages) & 1, &sh, p.status);
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        if (t == 1 && !active1) break;
+                        if (!ok_p) mbar_wait(&sh.p_full[t], (ph[t] + j) & 1, &sh, p.status);
+                        tc_fence_after();
+                        const uint32_t t_st = tmem + t * 256;
+                        const uint32_t dqt = dq_lo + t * kTile16;
+                        const uint32_t last_of_iter = (t == 1) ? 1u : (active1 ? 0u : 1u);
+                        // O_t (+)= P_t V_j
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk)
+                            mma_ts(t_st + 128, t_st + kk * 8, dvj + kk * (2048 >> 4), dv_hi, kIdescPV,
+                                   (kk > 0) || (j > 0));
+                        mma_commit_if(last_of_iter, &sh.kv_empty[sv]);
+                        // S_t = Q_t K_{j+1}^T (not after the last tile)
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            if (kk == 6) {
+                                if (t == 0 && active1) {
+                                    ok_p = mbar_test(&sh.p_full[1], (ph[1] + j) & 1);
+                                } else {
+                                    ok_v = mbar_test(next_v, next_v_par);
+                                    ok_k = mbar_test(next_k, next_k_par);
+                                    ok_p = mbar_test(&sh.p_full[0], (ph[0] + j + 1) & 1);
+                                }
+                            }
+                            const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
+                            mma_ss_if(more, t_st, dqt + off16, dkj + off16, dkm_hi, dkm_hi, kIdescQK, kk > 0);
+                        }
+                        mma_commit_if(more, &sh.s_full[t]);
+                        mma_commit_if(more & last_of_iter, &sh.kv_empty[sk]);
+                        // after the item's last Q K^T the Q buffer may take the next item's tiles
+                        mma_commit_if((j + 2 == n_tiles) & last_of_iter, &sh.q_empty);
+                    }
+                }
+                mma_commit(&sh.o_full);
+                u_glob += 2 * n_tiles;
+                ph[0] += n_tiles;
+                if (active1) ph[1] += n_tiles;
             }
-            mma_commit(&sh.o_full);
         }
       }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
         // ================= softmax / correction / epilogue =================
         const int t = warp >> 2;                        // which of the two tiles
-        if (t == 0 || active1) {
-            const int quarter = warp & 3;               // tensor-memory lanes this warp may touch
+        const int quarter = warp & 3;                   // tensor-memory lanes this warp may touch
+        const uint32_t t_s = tmem + ((uint32_t)(quarter * 32) << 16) + t * 256;
+        const uint32_t t_o = t_s + 128;
+        const float sc = p.scale_log2;
+        uint32_t ph = 0;                                // S/P tiles of this query tile handled so far
+        for (int k = 0;; ++k) {
+            if (!kPersistent && k > 0) break;
+            const int item_idx = kPersistent ? item_index(k, n_items) : (int)blockIdx.x;
+            if (item_idx < 0) break;
+            const Item it = get_item(p, item_idx);
+            if (t == 1 && !it.active1) continue;
+            const int n_tiles = it.n_tiles, r0 = it.r0, C = it.C, P = it.P, b = it.b, hg = it.hg, g0 = it.g0;
+            const TilePlan plan = it.plan;
             const int r = quarter * 32 + lane;          // query row inside the tile
             const int rr = r0 + r;                      // row inside the chunk
-            const uint32_t t_s = tmem + ((uint32_t)(quarter * 32) << 16) + t * 256;
-            const uint32_t t_o = t_s + 128;
             const int* pos = p.pos + (long long)b * p.ring;
             float m_used = -INFINITY, l_run = 0.f;
-            const float sc = p.scale_log2;
             for (int j = 0; j < n_tiles; ++j) {
                 bool is_chunk;
                 int start;
                 plan_tile(plan, j, is_chunk, start);
-                mbar_wait(&sh.s_full[t], j & 1, &sh, p.status);
+                mbar_wait(&sh.s_full[t], (ph + j) & 1, &sh, p.status);
                 tc_fence_after();
                 float s[128];
                 tmem_ld32(t_s + 0, s + 0);
@@ -665,43 +724,51 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
             }
 
             // ---- epilogue: O / l -> bf16 -> global ---------------------------------------------------
-            mbar_wait(&sh.o_full, 0, &sh, p.status);
+            ph += n_tiles;
+            mbar_wait(&sh.o_full, k & 1, &sh, p.status);
             tc_fence_after();
             const float inv = 1.f / l_run;
-            // Every MMA of this CTA has completed, so the tile's Q buffer is free: the warp stages its
-            // 32 rows there (16-byte pieces XOR-swizzled by row) and writes them out with every
-            // 256-byte row covered by 16 consecutive lanes, instead of one lane per row.
-            const uint32_t stage = sm_q + t * kTileBytes + (uint32_t)(quarter * 32) * 256;
+            // The warp stages 16 of its 32 rows at a time in its 4 KB of shared memory (16-byte pieces
+            // XOR-swizzled by row) and writes them out with every 256-byte row covered by 16
+            // consecutive lanes, instead of one lane per row.  (The Q buffers are not used for this:
+            // the producer may already be loading the next item's Q.)
+            const uint32_t stage = sm_epi + (uint32_t)(warp * 4096);
+            const int piece_r = lane & 15, half_r = lane >> 4;
+            const long long row0 = (long long)p.tok_off[b] + r0 + quarter * 32;
+            __nv_bfloat16* obase = p.out + (long long)(p.q_head0 + hg * p.G + g0 + t) * kD + piece_r * 8;
 #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                float o[32];
-                tmem_ld32(t_o + c * 32, o);
-                tmem_wait_ld();
+            for (int h = 0; h < 2; ++h) {
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    float o[32];
+                    tmem_ld32(t_o + c * 32, o);
+                    tmem_wait_ld();
+                    if ((lane >> 4) == h) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint32_t w0 = pack_bf16(o[8 * i + 0] * inv, o[8 * i + 1] * inv);
-                    const uint32_t w1 = pack_bf16(o[8 * i + 2] * inv, o[8 * i + 3] * inv);
-                    const uint32_t w2 = pack_bf16(o[8 * i + 4] * inv, o[8 * i + 5] * inv);
-                    const uint32_t w3 = pack_bf16(o[8 * i + 6] * inv, o[8 * i + 7] * inv);
-                    const uint32_t piece = (uint32_t)(c * 4 + i);
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + lane * 256 + ((piece ^ (lane & 15)) << 4)),
-                                 "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+                        for (int i = 0; i < 4; ++i) {
+                            const uint32_t w0 = pack_bf16(o[8 * i + 0] * inv, o[8 * i + 1] * inv);
+                            const uint32_t w1 = pack_bf16(o[8 * i + 2] * inv, o[8 * i + 3] * inv);
+                            const uint32_t w2 = pack_bf16(o[8 * i + 4] * inv, o[8 * i + 5] * inv);
+                            const uint32_t w3 = pack_bf16(o[8 * i + 6] * inv, o[8 * i + 7] * inv);
+                            const uint32_t piece = (uint32_t)(c * 4 + i);
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                                         ::"r"(stage + (lane & 15) * 256 + ((piece ^ (lane & 15)) << 4)),
+                                           "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+                        }
+                    }
                 }
-            }
-            __syncwarp();
-            {
-                const int piece = lane & 15, half = lane >> 4;
-                const long long row0 = (long long)p.tok_off[b] + r0 + quarter * 32;
-                __nv_bfloat16* obase = p.out + (long long)(p.q_head0 + hg * p.G + g0 + t) * kD + piece * 8;
+                __syncwarp();
 #pragma unroll 4
-                for (int i = 0; i < 16; ++i) {
-                    const int lr = 2 * i + half;                           // row inside the warp's 32
+                for (int i = 0; i < 8; ++i) {
+                    const int sr = 2 * i + half_r;                         // row inside the staged 16
+                    const int lr = 16 * h + sr;                            // row inside the warp's 32
                     uint32_t w0, w1, w2, w3;
                     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
-                                 : "r"(stage + lr * 256 + ((piece ^ (lr & 15)) << 4)) : "memory");
+                                 : "r"(stage + sr * 256 + ((piece_r ^ sr) << 4)) : "memory");
                     if (r0 + quarter * 32 + lr < C)
                         *reinterpret_cast<uint4*>(obase + (row0 + lr) * p.tok_stride) = make_uint4(w0, w1, w2, w3);
                 }
+                __syncwarp();
             }
         }
     }
@@ -717,16 +784,34 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
 
 }  // namespace
 
+static int g_num_sms = 0;
+
 cudaError_t prefill_setup() {
-    return cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(prefill_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 
 cudaError_t launch_prefill(const PrefillParams& p, const void* tq, const void* tk, const void* tv,
                            const void* ta, int n_items, cudaStream_t s) {
-    prefill_kernel<<<n_items, kThreads, kSmemBytes, s>>>(p, *static_cast<const CUtensorMap*>(tq),
-                                                        *static_cast<const CUtensorMap*>(tk),
-                                                        *static_cast<const CUtensorMap*>(tv),
-                                                        *static_cast<const CUtensorMap*>(ta));
+    PrefillParams pp = p;
+    pp.n_items = n_items;
+    if (p.kind == ZZ_KIND_STREAMING && g_num_sms > 0 && n_items > g_num_sms) {
+        // persistent CTAs, one per SM (tensor memory and shared memory allow no more)
+        prefill_kernel<true><<<g_num_sms, kThreads, kSmemBytes, s>>>(pp, *static_cast<const CUtensorMap*>(tq),
+                                                                   *static_cast<const CUtensorMap*>(tk),
+                                                                   *static_cast<const CUtensorMap*>(tv),
+                                                                   *static_cast<const CUtensorMap*>(ta));
+    } else {
+        prefill_kernel<false><<<n_items, kThreads, kSmemBytes, s>>>(pp, *static_cast<const CUtensorMap*>(tq),
+                                                                  *static_cast<const CUtensorMap*>(tk),
+                                                                  *static_cast<const CUtensorMap*>(tv),
+                                                                  *static_cast<const CUtensorMap*>(ta));
+    }
     count_launch();
     return cudaGetLastError();
 }
