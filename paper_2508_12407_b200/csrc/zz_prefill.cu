@@ -42,7 +42,7 @@ constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr uint32_t kAbortPolls = 1u << 10;
 constexpr float kRescaleThreshold = 8.f;    // log2 units of slack before O is rescaled
 #ifndef ZZ_POLY_EVERY
-#define ZZ_POLY_EVERY 4
+#define ZZ_POLY_EVERY 8
 #endif
 constexpr int kPolyEvery = ZZ_POLY_EVERY;   // one pair in kPolyEvery takes the polynomial exp2 (>= 17: none)
 
@@ -519,10 +519,24 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                         const uint32_t dqt = dq_lo + t * kTile16;
                         const uint32_t last_of_iter = (t == 1) ? 1u : (active1 ? 0u : 1u);
                         // O_t (+)= P_t V_j
+                        // all 24 descriptor words of the tile first, so that nothing but the MMAs
+                        // themselves sits between two MMAs
+                        uint32_t dvs[8], dqs[8], dks[8];
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
+                            dvs[kk] = dvj + kk * (2048 >> 4);
+                            dqs[kk] = dqt + off16;
+                            dks[kk] = dkj + off16;
+                        }
+                        asm volatile("" ::"r"(dvs[0]), "r"(dvs[1]), "r"(dvs[2]), "r"(dvs[3]), "r"(dvs[4]), "r"(dvs[5]),
+                                     "r"(dvs[6]), "r"(dvs[7]), "r"(dqs[0]), "r"(dqs[1]), "r"(dqs[2]), "r"(dqs[3]), "r"(dqs[4]),
+                                     "r"(dqs[5]), "r"(dqs[6]), "r"(dqs[7]), "r"(dks[0]), "r"(dks[1]), "r"(dks[2]), "r"(dks[3]),
+                                     "r"(dks[4]), "r"(dks[5]), "r"(dks[6]), "r"(dks[7])
+                                     : "memory");
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk)
-                            mma_ts(t_st + 128, t_st + kk * 8, dvj + kk * (2048 >> 4), dv_hi, kIdescPV,
-                                   (kk > 0) || (j > 0));
+                            mma_ts(t_st + 128, t_st + kk * 8, dvs[kk], dv_hi, kIdescPV, (kk > 0) || (j > 0));
                         mma_commit_if(last_of_iter, &sh.kv_empty[sv]);
                         // S_t = Q_t K_{j+1}^T (not after the last tile)
 #pragma unroll
@@ -536,8 +550,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                                     ok_p = mbar_test(&sh.p_full[0], (ph[0] + j + 1) & 1);
                                 }
                             }
-                            const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
-                            mma_ss_if(more, t_st, dqt + off16, dkj + off16, dkm_hi, dkm_hi, kIdescQK, kk > 0);
+                            mma_ss_if(more, t_st, dqs[kk], dks[kk], dkm_hi, dkm_hi, kIdescQK, kk > 0);
                         }
                         mma_commit_if(more, &sh.s_full[t]);
                         mma_commit_if(more & last_of_iter, &sh.kv_empty[sk]);
