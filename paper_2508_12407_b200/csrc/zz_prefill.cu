@@ -32,7 +32,8 @@ namespace {
 constexpr int kTile = 128;
 constexpr int kSubBytes = 128 * 128;        // [128 rows][64 bf16] sub-tile, 128-byte swizzled
 constexpr int kTileBytes = 2 * kSubBytes;   // a full [128][128] bf16 tile
-constexpr int kStages = 4;                  // ring of K and V tiles (K_0, V_0, K_1, V_1, ...)
+constexpr int kStages = 4;                  // K/V tiles held at once: two pair slots of (V_j, K_{j+1})
+constexpr int kPairs = 2;                   // one full / empty barrier per pair: what an iteration uses, it uses together
 constexpr int kThreads = 384;                // three warpgroups: softmax tile 0, softmax tile 1, TMA + MMA
 constexpr int kWarpTma = 8, kWarpMma = 9;
 constexpr int kRegsSoftmax = 208, kRegsAux = 88;   // 208 * 256 + 88 * 128 <= 65536 registers
@@ -53,8 +54,8 @@ constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);   // B (= V) is MN-major
 struct Shared {
     uint64_t q_full;
     uint64_t q_empty;          // the item's last Q K^T has completed: the Q buffer may be reloaded
-    uint64_t kv_full[kStages];
-    uint64_t kv_empty[kStages];
+    uint64_t kv_full[kPairs];
+    uint64_t kv_empty[kPairs];
     uint64_t s_full[2];
     uint64_t p_full[2];
     uint64_t o_full;
@@ -386,7 +387,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
     if (threadIdx.x == 0) {
         mbar_init(&sh.q_full, 1);
         mbar_init(&sh.q_empty, 1);
-        for (int i = 0; i < kStages; ++i) {
+        for (int i = 0; i < kPairs; ++i) {
             mbar_init(&sh.kv_full[i], 1);
             mbar_init(&sh.kv_empty[i], 1);
         }
@@ -415,7 +416,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
       if (warp == kWarpTma) {
         // ================= TMA producer =================
         if (lane == 0) {
-            uint32_t u_glob = 0;                      // K/V sub-tiles loaded so far (all items)
+            uint32_t u_glob = 0;                      // K/V pairs loaded so far (all items)
             for (int k = 0;; ++k) {
                 if (!kPersistent && k > 0) break;
                 const int idx = kPersistent ? item_index(k, n_items) : (int)blockIdx.x;
@@ -436,23 +437,29 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                     tma_load_3d(sm_q + kTileBytes, &tmap_q, 0, qh + 1, tok0 + it.r0, &sh.q_full);
                     tma_load_3d(sm_q + kTileBytes + kSubBytes, &tmap_q, 64, qh + 1, tok0 + it.r0, &sh.q_full);
                 }
-                for (int u = 0; u < 2 * it.n_tiles; ++u, ++u_glob) {
-                    const int stage = u_glob % kStages;
-                    mbar_wait(&sh.kv_empty[stage], ((u_glob / kStages) & 1) ^ 1, &sh, p.status);
-                    bool is_chunk;
-                    int start;
-                    plan_tile(it.plan, u >> 1, is_chunk, start);
-                    const bool is_v = u & 1;
-                    const uint32_t dst = sm_kv + stage * kTileBytes;
-                    mbar_expect_tx(&sh.kv_full[stage], kTileBytes);
-                    if (is_chunk) {
-                        const CUtensorMap* m = is_v ? &tmap_v : &tmap_k;
-                        tma_load_3d(dst, m, 0, src_head, tok0 + start, &sh.kv_full[stage]);
-                        tma_load_3d(dst + kSubBytes, m, 64, src_head, tok0 + start, &sh.kv_full[stage]);
-                    } else {
-                        const int row = (is_v ? v_row0 : k_row0) + start;
-                        tma_load_2d(dst, &tmap_arena, 0, row, &sh.kv_full[stage]);
-                        tma_load_2d(dst + kSubBytes, &tmap_arena, 64, row, &sh.kv_full[stage]);
+                // pair pi of the item: pi = 0 holds K_0 alone, pi = j + 1 holds (V_j, K_{j+1}), the last one
+                // V_{n-1} alone; slot = running pair count % 2, V in the slot's first tile, K in its second
+                for (int pi = 0; pi <= it.n_tiles; ++pi, ++u_glob) {
+                    const int slot = u_glob % kPairs;
+                    mbar_wait(&sh.kv_empty[slot], ((u_glob / kPairs) & 1) ^ 1, &sh, p.status);
+                    const bool has_v = pi > 0, has_k = pi < it.n_tiles;
+                    mbar_expect_tx(&sh.kv_full[slot], (has_v && has_k) ? 2 * kTileBytes : kTileBytes);
+#pragma unroll
+                    for (int is_k = 0; is_k < 2; ++is_k) {
+                        if (is_k ? !has_k : !has_v) continue;
+                        bool is_chunk;
+                        int start;
+                        plan_tile(it.plan, is_k ? pi : pi - 1, is_chunk, start);
+                        const uint32_t dst = sm_kv + (slot * 2 + is_k) * kTileBytes;
+                        if (is_chunk) {
+                            const CUtensorMap* m = is_k ? &tmap_k : &tmap_v;
+                            tma_load_3d(dst, m, 0, src_head, tok0 + start, &sh.kv_full[slot]);
+                            tma_load_3d(dst + kSubBytes, m, 64, src_head, tok0 + start, &sh.kv_full[slot]);
+                        } else {
+                            const int row = (is_k ? k_row0 : v_row0) + start;
+                            tma_load_2d(dst, &tmap_arena, 0, row, &sh.kv_full[slot]);
+                            tma_load_2d(dst + kSubBytes, &tmap_arena, 64, row, &sh.kv_full[slot]);
+                        }
                     }
                 }
             }
@@ -467,7 +474,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
             const uint32_t dkm_hi = (uint32_t)(dq >> 32), dv_hi = (uint32_t)(dv >> 32);
             constexpr uint32_t kTile16 = kTileBytes >> 4;
             // Counters that run across the items of this CTA (barrier phases never restart):
-            uint32_t u_glob = 0;          // K/V sub-tiles consumed
+            uint32_t u_glob = 0;          // K/V pairs consumed
             uint32_t ph[2] = {0, 0};      // S/P tiles handled per query tile (tile 1 only in items that have it)
             for (int k = 0;; ++k) {
                 if (!kPersistent && k > 0) break;
@@ -478,7 +485,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                 const bool active1 = it.active1;
                 const int n_act = active1 ? 2 : 1;
                 mbar_wait(&sh.q_full, k & 1, &sh, p.status);
-                mbar_wait(&sh.kv_full[u_glob % kStages], (u_glob / kStages) & 1, &sh, p.status);
+                mbar_wait(&sh.kv_full[u_glob % kPairs], (u_glob / kPairs) & 1, &sh, p.status);
                 tc_fence_after();
                 // S_t = Q_t K_0^T
                 for (int t = 0; t < n_act; ++t) {
@@ -486,30 +493,26 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                     for (int kk = 0; kk < 8; ++kk) {
                         const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
                         mma_ss(tmem + t * 256, dq_lo + t * kTile16 + off16,
-                               dk_lo + (u_glob % kStages) * kTile16 + off16, dkm_hi, dkm_hi, kIdescQK, kk > 0);
+                               dk_lo + ((u_glob % kPairs) * 2 + 1) * kTile16 + off16, dkm_hi, dkm_hi, kIdescQK, kk > 0);
                     }
                     mma_commit(&sh.s_full[t]);
                 }
-                mma_commit(&sh.kv_empty[u_glob % kStages]);
-                mma_commit_if(n_tiles == 1, &sh.q_empty);
+                mma_commit(&sh.kv_empty[u_glob % kPairs]);
+                if (kPersistent) mma_commit_if(n_tiles == 1, &sh.q_empty);
                 // The thread that issues tcgen05.mma is held at each one until the tensor pipe has room,
                 // so whatever it does between two tiles leaves the pipe idle.  The barriers of the next
                 // tile (K/V stages, the other tile's P) are therefore probed, without blocking, two MMAs
                 // before the current tile's last one; the probe's latency then overlaps those MMAs, and
                 // the blocking wait is only entered when a probe came back negative.
-                bool ok_v = false, ok_k = false, ok_p = false;
+                bool ok_kv = false, ok_p = false;
                 for (int j = 0; j < n_tiles; ++j) {
-                    const uint32_t uv = u_glob + 2 * j + 1, uk = u_glob + 2 * j + 2;
-                    const uint32_t sv = uv % kStages, sk = uk % kStages;
+                    const uint32_t pj = u_glob + 1 + j;             // the pair (V_j, K_{j+1})
+                    const uint32_t slot = pj % kPairs;
                     const uint32_t more = (j + 1) < n_tiles;
-                    const uint32_t dvj = dv_lo + sv * kTile16, dkj = dk_lo + sk * kTile16;
-                    // barriers of the next iteration (valid addresses and parities even past the end)
-                    const uint32_t uv2 = uv + 2, uk2 = uk + 2;
-                    uint64_t* next_v = &sh.kv_full[uv2 % kStages];
-                    uint64_t* next_k = &sh.kv_full[uk2 % kStages];
-                    const uint32_t next_v_par = (uv2 / kStages) & 1, next_k_par = (uk2 / kStages) & 1;
-                    if (!ok_v) mbar_wait(&sh.kv_full[sv], (uv / kStages) & 1, &sh, p.status);
-                    if (!ok_k && more) mbar_wait(&sh.kv_full[sk], (uk / kStages) & 1, &sh, p.status);
+                    const uint32_t dvj = dv_lo + (slot * 2) * kTile16, dkj = dk_lo + (slot * 2 + 1) * kTile16;
+                    uint64_t* next_kv = &sh.kv_full[(pj + 1) % kPairs];
+                    const uint32_t next_kv_par = ((pj + 1) / kPairs) & 1;
+                    if (!ok_kv) mbar_wait(&sh.kv_full[slot], (pj / kPairs) & 1, &sh, p.status);
 #pragma unroll
                     for (int t = 0; t < 2; ++t) {
                         if (t == 1 && !active1) break;
@@ -518,7 +521,6 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                         const uint32_t t_st = tmem + t * 256;
                         const uint32_t dqt = dq_lo + t * kTile16;
                         const uint32_t last_of_iter = (t == 1) ? 1u : (active1 ? 0u : 1u);
-                        // O_t (+)= P_t V_j
                         // all 24 descriptor words of the tile first, so that nothing but the MMAs
                         // themselves sits between two MMAs
                         uint32_t dvs[8], dqs[8], dks[8];
@@ -534,32 +536,34 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                                      "r"(dqs[5]), "r"(dqs[6]), "r"(dqs[7]), "r"(dks[0]), "r"(dks[1]), "r"(dks[2]), "r"(dks[3]),
                                      "r"(dks[4]), "r"(dks[5]), "r"(dks[6]), "r"(dks[7])
                                      : "memory");
+                        // O_t (+)= P_t V_j
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk)
                             mma_ts(t_st + 128, t_st + kk * 8, dvs[kk], dv_hi, kIdescPV, (kk > 0) || (j > 0));
-                        mma_commit_if(last_of_iter, &sh.kv_empty[sv]);
                         // S_t = Q_t K_{j+1}^T (not after the last tile)
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
                             if (kk == 6) {
+                                // non-blocking probes of what is issued next
                                 if (t == 0 && active1) {
                                     ok_p = mbar_test(&sh.p_full[1], (ph[1] + j) & 1);
                                 } else {
-                                    ok_v = mbar_test(next_v, next_v_par);
-                                    ok_k = mbar_test(next_k, next_k_par);
+                                    ok_kv = mbar_test(next_kv, next_kv_par);
                                     ok_p = mbar_test(&sh.p_full[0], (ph[0] + j + 1) & 1);
                                 }
                             }
                             mma_ss_if(more, t_st, dqs[kk], dks[kk], dkm_hi, dkm_hi, kIdescQK, kk > 0);
                         }
+                        // Commits cost tensor-pipe time beyond the first one after an MMA group, so there
+                        // is one per tile (its S) plus one per iteration (the K/V pair is free again)
                         mma_commit_if(more, &sh.s_full[t]);
-                        mma_commit_if(more & last_of_iter, &sh.kv_empty[sk]);
+                        mma_commit_if(last_of_iter, &sh.kv_empty[slot]);
                         // after the item's last Q K^T the Q buffer may take the next item's tiles
-                        mma_commit_if((j + 2 == n_tiles) & last_of_iter, &sh.q_empty);
+                        if (kPersistent) mma_commit_if((j + 2 == n_tiles) & last_of_iter, &sh.q_empty);
                     }
                 }
                 mma_commit(&sh.o_full);
-                u_glob += 2 * n_tiles;
+                u_glob += n_tiles + 1;
                 ph[0] += n_tiles;
                 if (active1) ph[1] += n_tiles;
             }
