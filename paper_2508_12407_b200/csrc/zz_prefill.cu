@@ -466,10 +466,18 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
         }
       } else if (warp == kWarpMma) {
         // ================= MMA issuer =================
-        if (lane == 0) {
+        // The whole warp runs this loop and its barrier waits; one lane issues the MMAs and commits.
+        // Measured on this hardware: an issuing thread that sits alone in a divergent branch is
+        // starved of issue slots by the softmax warps of its SM sub-partition (a tile's 16 MMAs took
+        // up to 3x their 1024 cycles next to a busy warp), a warp in uniform control flow is not
+        // (1.1x).  Everything the descriptors derive from is made provably warp-uniform for the
+        // same reason.
+        {
+            const bool leader = lane == 0;
+            const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
             const uint64_t dq = make_desc(sm_q, 16, 1024);          // Q tile 0, K-major
-            const uint64_t dk = make_desc(sm_kv, 16, 1024);         // K tile in stage 0, K-major
-            const uint64_t dv = make_desc(sm_kv, kSubBytes, 1024);  // V tile in stage 0, MN-major
+            const uint64_t dk = make_desc(sm_kv, 16, 1024);         // K tile of pair slot 0, K-major
+            const uint64_t dv = make_desc(sm_kv, kSubBytes, 1024);  // V tile of pair slot 0, MN-major
             const uint32_t dq_lo = (uint32_t)dq, dk_lo = (uint32_t)dk, dv_lo = (uint32_t)dv;
             const uint32_t dkm_hi = (uint32_t)(dq >> 32), dv_hi = (uint32_t)(dv >> 32);
             constexpr uint32_t kTile16 = kTileBytes >> 4;
@@ -481,88 +489,65 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                 const int idx = kPersistent ? item_index(k, n_items) : (int)blockIdx.x;
                 if (idx < 0) break;
                 const Item it = get_item(p, idx);
-                const int n_tiles = it.n_tiles;
+                const int n_tiles = __shfl_sync(0xffffffffu, it.n_tiles, 0);
                 const bool active1 = it.active1;
                 const int n_act = active1 ? 2 : 1;
                 mbar_wait(&sh.q_full, k & 1, &sh, p.status);
                 mbar_wait(&sh.kv_full[u_glob % kPairs], (u_glob / kPairs) & 1, &sh, p.status);
                 tc_fence_after();
-                // S_t = Q_t K_0^T
-                for (int t = 0; t < n_act; ++t) {
+                if (leader) {
+                    // S_t = Q_t K_0^T
+                    for (int t = 0; t < n_act; ++t) {
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
-                        mma_ss(tmem + t * 256, dq_lo + t * kTile16 + off16,
-                               dk_lo + ((u_glob % kPairs) * 2 + 1) * kTile16 + off16, dkm_hi, dkm_hi, kIdescQK, kk > 0);
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
+                            mma_ss(tmem_u + t * 256, dq_lo + t * kTile16 + off16,
+                                   dk_lo + ((u_glob % kPairs) * 2 + 1) * kTile16 + off16, dkm_hi, dkm_hi, kIdescQK, kk > 0);
+                        }
+                        mma_commit(&sh.s_full[t]);
                     }
-                    mma_commit(&sh.s_full[t]);
+                    mma_commit(&sh.kv_empty[u_glob % kPairs]);
+                    if (kPersistent) mma_commit_if(n_tiles == 1, &sh.q_empty);
                 }
-                mma_commit(&sh.kv_empty[u_glob % kPairs]);
-                if (kPersistent) mma_commit_if(n_tiles == 1, &sh.q_empty);
-                // The thread that issues tcgen05.mma is held at each one until the tensor pipe has room,
-                // so whatever it does between two tiles leaves the pipe idle.  The barriers of the next
-                // tile (K/V stages, the other tile's P) are therefore probed, without blocking, two MMAs
-                // before the current tile's last one; the probe's latency then overlaps those MMAs, and
-                // the blocking wait is only entered when a probe came back negative.
-                bool ok_kv = false, ok_p = false;
+                __syncwarp();
                 for (int j = 0; j < n_tiles; ++j) {
                     const uint32_t pj = u_glob + 1 + j;             // the pair (V_j, K_{j+1})
                     const uint32_t slot = pj % kPairs;
                     const uint32_t more = (j + 1) < n_tiles;
                     const uint32_t dvj = dv_lo + (slot * 2) * kTile16, dkj = dk_lo + (slot * 2 + 1) * kTile16;
-                    uint64_t* next_kv = &sh.kv_full[(pj + 1) % kPairs];
-                    const uint32_t next_kv_par = ((pj + 1) / kPairs) & 1;
-                    if (!ok_kv) mbar_wait(&sh.kv_full[slot], (pj / kPairs) & 1, &sh, p.status);
+                    mbar_wait(&sh.kv_full[slot], (pj / kPairs) & 1, &sh, p.status);
 #pragma unroll
                     for (int t = 0; t < 2; ++t) {
                         if (t == 1 && !active1) break;
-                        if (!ok_p) mbar_wait(&sh.p_full[t], (ph[t] + j) & 1, &sh, p.status);
+                        mbar_wait(&sh.p_full[t], (ph[t] + j) & 1, &sh, p.status);
                         tc_fence_after();
-                        const uint32_t t_st = tmem + t * 256;
-                        const uint32_t dqt = dq_lo + t * kTile16;
-                        const uint32_t last_of_iter = (t == 1) ? 1u : (active1 ? 0u : 1u);
-                        // all 24 descriptor words of the tile first, so that nothing but the MMAs
-                        // themselves sits between two MMAs
-                        uint32_t dvs[8], dqs[8], dks[8];
+                        if (leader) {
+                            const uint32_t t_st = tmem_u + t * 256;
+                            const uint32_t dqt = dq_lo + t * kTile16;
+                            const uint32_t last_of_iter = (t == 1) ? 1u : (active1 ? 0u : 1u);
+                            // O_t (+)= P_t V_j
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
-                            dvs[kk] = dvj + kk * (2048 >> 4);
-                            dqs[kk] = dqt + off16;
-                            dks[kk] = dkj + off16;
-                        }
-                        asm volatile("" ::"r"(dvs[0]), "r"(dvs[1]), "r"(dvs[2]), "r"(dvs[3]), "r"(dvs[4]), "r"(dvs[5]),
-                                     "r"(dvs[6]), "r"(dvs[7]), "r"(dqs[0]), "r"(dqs[1]), "r"(dqs[2]), "r"(dqs[3]), "r"(dqs[4]),
-                                     "r"(dqs[5]), "r"(dqs[6]), "r"(dqs[7]), "r"(dks[0]), "r"(dks[1]), "r"(dks[2]), "r"(dks[3]),
-                                     "r"(dks[4]), "r"(dks[5]), "r"(dks[6]), "r"(dks[7])
-                                     : "memory");
-                        // O_t (+)= P_t V_j
+                            for (int kk = 0; kk < 8; ++kk)
+                                mma_ts(t_st + 128, t_st + kk * 8, dvj + kk * (2048 >> 4), dv_hi, kIdescPV,
+                                       (kk > 0) || (j > 0));
+                            // S_t = Q_t K_{j+1}^T (not after the last tile)
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk)
-                            mma_ts(t_st + 128, t_st + kk * 8, dvs[kk], dv_hi, kIdescPV, (kk > 0) || (j > 0));
-                        // S_t = Q_t K_{j+1}^T (not after the last tile)
-#pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            if (kk == 6) {
-                                // non-blocking probes of what is issued next
-                                if (t == 0 && active1) {
-                                    ok_p = mbar_test(&sh.p_full[1], (ph[1] + j) & 1);
-                                } else {
-                                    ok_kv = mbar_test(next_kv, next_kv_par);
-                                    ok_p = mbar_test(&sh.p_full[0], (ph[0] + j + 1) & 1);
-                                }
+                            for (int kk = 0; kk < 8; ++kk) {
+                                const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
+                                mma_ss_if(more, t_st, dqt + off16, dkj + off16, dkm_hi, dkm_hi, kIdescQK, kk > 0);
                             }
-                            mma_ss_if(more, t_st, dqs[kk], dks[kk], dkm_hi, dkm_hi, kIdescQK, kk > 0);
+                            // Commits cost tensor-pipe time beyond the first one after an MMA group, so
+                            // there is one per tile (its S) plus one per iteration (the K/V pair is free)
+                            mma_commit_if(more, &sh.s_full[t]);
+                            mma_commit_if(last_of_iter, &sh.kv_empty[slot]);
+                            // after the item's last Q K^T the Q buffer may take the next item's tiles
+                            if (kPersistent) mma_commit_if((j + 2 == n_tiles) & last_of_iter, &sh.q_empty);
                         }
-                        // Commits cost tensor-pipe time beyond the first one after an MMA group, so there
-                        // is one per tile (its S) plus one per iteration (the K/V pair is free again)
-                        mma_commit_if(more, &sh.s_full[t]);
-                        mma_commit_if(last_of_iter, &sh.kv_empty[slot]);
-                        // after the item's last Q K^T the Q buffer may take the next item's tiles
-                        if (kPersistent) mma_commit_if((j + 2 == n_tiles) & last_of_iter, &sh.q_empty);
+                        __syncwarp();
                     }
                 }
-                mma_commit(&sh.o_full);
+                if (leader) mma_commit(&sh.o_full);
+                __syncwarp();
                 u_glob += n_tiles + 1;
                 ph[0] += n_tiles;
                 if (active1) ph[1] += n_tiles;
