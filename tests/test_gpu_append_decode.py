@@ -110,6 +110,44 @@ def test_ragged_batch():
     run_append_decode(2, 5, 8, 2, 16, 48, [1, 0], lens, 5, seed=9, chunk_cap=1500)
 
 
+def test_maximum_batch():
+    # ZZ_MAX_BATCH sequences, ragged from 1 token upwards, several of them shorter than the ring
+    rng = np.random.default_rng(64)
+    lens = [int(x) for x in rng.integers(1, 700, size=binding.ZZ_MAX_BATCH)]
+    lens[0], lens[1], lens[-1] = 1, 2, 699
+    run_append_decode(2, binding.ZZ_MAX_BATCH, 8, 2, 16, 48, [1, 0], lens, 2, seed=64, chunk_cap=700)
+
+
+def test_store_filled_to_capacity_exactly():
+    # the last decode step lands on the last slot of every retrieval store; one more is refused
+    import torch
+    D, B = 128, 2
+    lens = [130, 257]
+    cap = [n + 1 for n in lens]
+    cache = make(1, B, 4, 1, 8, 8, [1], cap)
+    w = inputs.Workload("t", 1, B, 4, 1, D, 8, 8, 1, 0, 0, 1, seed=5)
+    for b in range(B):
+        pass
+    ks = np.concatenate([inputs.qkv_bf16(w, 0, b, 0, lens[b])[1] for b in range(B)])
+    vs = np.concatenate([inputs.qkv_bf16(w, 0, b, 0, lens[b])[2] for b in range(B)])
+    cache.kv_append(0, to_dev(ks), to_dev(vs), lens)
+    q = to_dev(np.concatenate([inputs.qkv_bf16(w, 0, b, lens[b], 1)[0] for b in range(B)]))
+    k = to_dev(np.concatenate([inputs.qkv_bf16(w, 0, b, lens[b], 1)[1] for b in range(B)]))
+    v = to_dev(np.concatenate([inputs.qkv_bf16(w, 0, b, lens[b], 1)[2] for b in range(B)]))
+    out = torch.zeros_like(q)
+    cache.decode_step(0, q, k, v, out)                       # fills the last slot
+    assert [cache.len(0, b) for b in range(B)] == cap
+    with pytest.raises(binding.ZigzagError) as e:
+        cache.decode_step(0, q, k, v, out)
+    assert e.value.status == binding.ZZ_ERR_CAPACITY
+    with pytest.raises(binding.ZigzagError) as e:
+        cache.decode_step_all(q.view(1, B, 4, D), k.view(1, B, 1, D), v.view(1, B, 1, D), out.view(1, B, 4, D))
+    assert e.value.status == binding.ZZ_ERR_CAPACITY
+    assert [cache.export(0, b, binding.KIND_RETRIEVAL)[3] for b in range(B)] == cap
+    assert cache.last_status() == 0
+    cache.close()
+
+
 def test_min_chunk_tuning_keeps_results():
     D = 128
     w = inputs.Workload("t", 1, 1, 8, 2, D, 8, 8, 1, 0, 0, 1, seed=77)

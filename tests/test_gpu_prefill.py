@@ -120,6 +120,15 @@ def test_ragged_batch_packed():
     run_prefill(2, 4, 8, 2, 32, 96, [1, 0], plans, seed=50, n_decode=2)
 
 
+def test_maximum_batch_packed_prefill():
+    # ZZ_MAX_BATCH sequences in one packed call, some of them absent from a round
+    rng = np.random.default_rng(65)
+    plans = [[int(rng.integers(0, 200)), int(rng.integers(1, 150))] for _ in range(binding.ZZ_MAX_BATCH)]
+    plans[0] = [0, 1]
+    plans[1] = [129, 0]
+    run_prefill(2, binding.ZZ_MAX_BATCH, 4, 2, 8, 24, [1, 0], plans, seed=65, n_decode=1)
+
+
 def test_decode_step_equals_prefill_row():
     # the last row of a prefill and a decode step at the same position agree within tolerance
     D, S, W, n = 128, 32, 64, 500
