@@ -108,11 +108,13 @@ int zz_cache_len(const zz_cache_t* cache, int layer, int seq, int32_t* len);
  * (fewest tokens per split of the long-store decode plan; a multiple of 16, default 256);
  * "decode_short_tokens" (tokens per CTA of the short-store plan, and the threshold
  * total_tokens * kv_heads <= SMs * value below which it is used; multiple of 16, default
- * 384; 0 disables the short-store plan); "decode_overlap" (how the per-layer
- * launches of zz_decode_step_all follow one another.  2, the default: programmatic dependent launch
- * and no wait between layers -- they share no scratch, so a layer's kernel fills the SMs the
- * previous one leaves idle; 1: the same, but each kernel waits for the previous one before it
- * merges; 0: plain stream order). */
+ * 384; 0 disables the short-store plan); "decode_overlap" (how the layers
+ * of zz_decode_step_all are launched.  3, the default: all exclusive retrieval layers in one
+ * launch and all exclusive streaming layers in another (possible when no layer is mixed and all
+ * layers hold equally long sequences; otherwise as 2); 2: one launch per layer, programmatic
+ * dependent launch and no wait between layers -- they share no scratch, so a layer's kernel fills
+ * the SMs the previous one leaves idle; 1: the same, but each kernel waits for the previous one
+ * before it merges; 0: plain stream order). */
 int zz_tune(zz_cache_t* cache, const char* key, int value);
 
 /* KV append with sink + recent eviction (paper: Introduction -- the KV cache grows with

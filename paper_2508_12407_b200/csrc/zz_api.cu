@@ -63,7 +63,7 @@ size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 struct Layout {
     // workspace sections (byte offsets)
     size_t off_status, off_len, off_pos, off_desc, off_heads, off_counters, off_part_ml, off_part_o,
-        off_qc, off_oc, work_bytes;
+        off_qc, off_oc, off_layer_ids, work_bytes;
     size_t arena_bytes, counters_per_layer, items_per_layer;
 };
 
@@ -123,6 +123,8 @@ struct zz_cache {
     std::vector<int> cap;             // [B]
     std::vector<int> len;             // [L*B] host mirror
     std::vector<SeqDesc> desc;        // [L*B]
+    std::vector<int> layer_ids;       // exclusive retrieval layers (ascending), then exclusive streaming layers
+    int n_excl_R, n_excl_S;
     Layout lay;
     unsigned char* arena;
     unsigned char* work;
@@ -140,6 +142,7 @@ struct zz_cache {
     int* d_len(int l) const { return reinterpret_cast<int*>(work + lay.off_len) + (size_t)l * B; }
     int* d_pos(int l) const { return reinterpret_cast<int*>(work + lay.off_pos) + (size_t)l * B * ring; }
     SeqDesc* d_desc(int l) const { return reinterpret_cast<SeqDesc*>(work + lay.off_desc) + (size_t)l * B; }
+    int* d_layer_ids() const { return reinterpret_cast<int*>(work + lay.off_layer_ids); }
     int* d_heads(int l) const { return reinterpret_cast<int*>(work + lay.off_heads) + (size_t)l * Hkv; }
     unsigned int* d_counters(int l) const {
         return reinterpret_cast<unsigned int*>(work + lay.off_counters) + (size_t)l * lay.counters_per_layer;
@@ -216,6 +219,7 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
     lay->off_pos = w; w += align_up((size_t)L * B * ring * sizeof(int));
     lay->off_desc = w; w += align_up((size_t)L * B * sizeof(SeqDesc));
     lay->off_heads = w; w += align_up((size_t)L * Hkv * sizeof(int));
+    lay->off_layer_ids = w; w += align_up((size_t)L * sizeof(int));
     // per layer: arrival counters and the split partials of the layer's launches, indexed by work
     // item (at most kMaxSlots + B * Hkv items per launch), so that the launches of different
     // layers share no scratch and may overlap
@@ -277,7 +281,8 @@ void plan_splits(const zz_cache* c, const int* n, int Hg, int* warps, int* chunk
 // k_new/v_new != nullptr: fused append of one token per sequence (host lengths not yet bumped)
 int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q, __nv_bfloat16* out,
                         int q_head0, cudaStream_t st, const __nv_bfloat16* k_new = nullptr,
-                        const __nv_bfloat16* v_new = nullptr, int bump_len = 0, int overlap = 0) {
+                        const __nv_bfloat16* v_new = nullptr, int bump_len = 0, int overlap = 0,
+                        const int* d_layer_ids = nullptr, int n_multi = 1) {
     const int Hg = (kind == ZZ_KIND_RETRIEVAL) ? c->nR[layer] : c->Hkv - c->nR[layer];
     if (Hg == 0) return ZZ_OK;
     zz::DecodeParams p;
@@ -325,7 +330,26 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
     // another launch of the same independent chain may follow.
     if (c->last_nowait && overlap != 2) overlap = 0;
     c->last_nowait = (overlap == 2);
-    const cudaError_t e = zz::launch_decode(p, items, warps, st, overlap);
+    if (d_layer_ids) {
+        // one launch for n_multi layers with identical lengths: `layer` stands for all of them in the
+        // plan above; every per-layer pointer becomes the layer-0 pointer plus a stride per layer
+        p.layer_ids = d_layer_ids;
+        p.desc_table = c->d_desc(0);
+        p.len = c->d_len(0);
+        p.pos = c->d_pos(0);
+        p.head_list = c->d_heads(0);
+        p.counters = c->d_counters(0);
+        p.seq_counters = c->d_counters(0) + (size_t)c->B * c->Hkv;
+        p.part_o = c->d_part_o(0);
+        p.part_ml = c->d_part_ml(0);
+        p.st_len = c->B;
+        p.st_pos = (long long)c->B * c->ring;
+        p.st_q = (long long)c->B * c->Hq * kD;
+        p.st_kv = (long long)c->B * c->Hkv * kD;
+        p.st_cnt = (long long)c->lay.counters_per_layer;
+        p.st_part = (long long)c->lay.items_per_layer * c->G;
+    }
+    const cudaError_t e = zz::launch_decode(p, items, warps, st, overlap, n_multi);
     zz::prof_end(pk, st);
     return e == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
 }
@@ -440,7 +464,7 @@ int zz_cache_create(const zz_config_t* cfg, void* d_arena, size_t arena_bytes, v
     c->max_new = cfg->max_new_tokens; c->scale = cfg->softmax_scale;
     c->decode_min_chunk = 256;
     c->decode_short_tokens = 384;
-    c->decode_overlap = 2;
+    c->decode_overlap = 3;
     c->last_nowait = false;
     compute_layout(cfg, &c->lay, &c->desc);
     if (arena_bytes < c->lay.arena_bytes || workspace_bytes < c->lay.work_bytes) {
@@ -467,6 +491,12 @@ int zz_cache_create(const zz_config_t* cfg, void* d_arena, size_t arena_bytes, v
         }
         if (r > 0 && r < c->Hkv) c->has_mixed = true;
     }
+    c->n_excl_R = c->n_excl_S = 0;
+    for (int l = 0; l < c->L; ++l)
+        if (c->nR[l] == c->Hkv) { c->layer_ids.push_back(l); ++c->n_excl_R; }
+    for (int l = 0; l < c->L; ++l)
+        if (c->nR[l] == 0) { c->layer_ids.push_back(l); ++c->n_excl_S; }
+    c->layer_ids.resize(c->L, 0);
     c->cap.assign(cfg->capacity, cfg->capacity + c->B);
     c->len.assign((size_t)c->L * c->B, 0);
 
@@ -483,6 +513,9 @@ int zz_cache_create(const zz_config_t* cfg, void* d_arena, size_t arena_bytes, v
                        cudaMemcpyHostToDevice);
     if (e == cudaSuccess)
         e = cudaMemcpy(c->work + c->lay.off_heads, c->heads.data(), c->heads.size() * sizeof(int),
+                       cudaMemcpyHostToDevice);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(c->work + c->lay.off_layer_ids, c->layer_ids.data(), c->layer_ids.size() * sizeof(int),
                        cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
@@ -526,7 +559,7 @@ int zz_tune(zz_cache_t* c, const char* key, int value) {
         return ZZ_OK;
     }
     if (!strcmp(key, "decode_overlap")) {
-        if (value < 0 || value > 2) return ZZ_ERR_INVALID_ARG;
+        if (value < 0 || value > 3) return ZZ_ERR_INVALID_ARG;
         c->decode_overlap = value;
         return ZZ_OK;
     }
@@ -635,7 +668,8 @@ static int decode_step_impl(zz_cache_t* c, int layer, const void* d_q, const voi
     int r;
     if (!c->mixed(layer)) {
         const int kind = nR ? ZZ_KIND_RETRIEVAL : ZZ_KIND_STREAMING;
-        r = launch_decode_group(c, layer, kind, q, out, 0, st, k, v, 1, overlap ? c->decode_overlap : (c->decode_overlap ? 3 : 0));
+        r = launch_decode_group(c, layer, kind, q, out, 0, st, k, v, 1,
+                                overlap ? (c->decode_overlap > 2 ? 2 : c->decode_overlap) : (c->decode_overlap ? 3 : 0));
     } else {
         r = regroup(c, layer, q, c->d_qc(), c->B, 1, st);
         const int ov = c->decode_overlap ? 3 : 0;
@@ -657,6 +691,36 @@ int zz_decode_step_all(zz_cache_t* c, const void* d_q, const void* d_k, const vo
     for (int l = 0; l < c->L; ++l)
         for (int b = 0; b < c->B; ++b)
             if (c->nR[l] > 0 && c->len[(size_t)l * c->B + b] + 1 > c->cap[b]) return ZZ_ERR_CAPACITY;
+    // All layers exclusive and of equal lengths: one launch for the retrieval layers and one for the
+    // streaming layers (blockIdx.y = layer).  The layers are independent (own stores, lengths,
+    // scratch and output slice; q/k/v of all layers are inputs of the call), so a launch over many
+    // layers only removes launch boundaries: no ramp-up and tail per layer, and the ~3 us per launch
+    // that a streaming layer's few CTAs cannot fill.
+    bool same_len = !c->has_mixed && c->decode_overlap == 3;
+    for (int l = 1; l < c->L && same_len; ++l)
+        for (int b = 0; b < c->B; ++b)
+            if (c->len[(size_t)l * c->B + b] != c->len[b]) same_len = false;
+    if (same_len) {
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        if (((uintptr_t)d_q | (uintptr_t)d_k | (uintptr_t)d_v | (uintptr_t)d_out) & 15) return ZZ_ERR_INVALID_ARG;
+        const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(d_q);
+        const __nv_bfloat16* k = static_cast<const __nv_bfloat16*>(d_k);
+        const __nv_bfloat16* v = static_cast<const __nv_bfloat16*>(d_v);
+        __nv_bfloat16* out = static_cast<__nv_bfloat16*>(d_out);
+        int r = ZZ_OK;
+        bool first = true;
+        if (c->n_excl_R > 0) {
+            r = launch_decode_group(c, c->layer_ids[0], ZZ_KIND_RETRIEVAL, q, out, 0, st, k, v, 1, 0, c->d_layer_ids(),
+                                    c->n_excl_R);
+            first = false;
+        }
+        if (r == ZZ_OK && c->n_excl_S > 0)
+            r = launch_decode_group(c, c->layer_ids[c->n_excl_R], ZZ_KIND_STREAMING, q, out, 0, st, k, v, 1,
+                                    first ? 0 : 2, c->d_layer_ids() + c->n_excl_R, c->n_excl_S);
+        if (r != ZZ_OK) return r;
+        for (size_t i = 0; i < c->len.size(); ++i) c->len[i] += 1;
+        return ZZ_OK;
+    }
     for (int l = 0; l < c->L; ++l) {
         // q/k/v of every layer are inputs of this call, and layer l's launch reads nothing that layer
         // l-1's launches write before its griddepcontrol.wait, so consecutive layers may overlap

@@ -69,6 +69,12 @@ struct DecodeParams {
     int split_start[ZZ_MAX_BATCH + 1];  // prefix sum of per-sequence split counts
     int chunk[ZZ_MAX_BATCH];            // tokens per split of each sequence
     SeqDesc sd[ZZ_MAX_BATCH];           // store addresses of every sequence of this layer
+    // several layers in one launch (blockIdx.y): layer_ids[y] is the layer, every per-layer pointer
+    // above is then the layer-0 pointer and advances by these strides (elements) per layer; the
+    // store addresses come from desc_table[layer * B + b].  layer_ids == nullptr: one layer.
+    const int* layer_ids;
+    const SeqDesc* desc_table;
+    long long st_len, st_pos, st_q, st_kv, st_cnt, st_part;
 };
 
 struct GatherParams {
@@ -105,7 +111,7 @@ struct PrefillParams {
 
 // ---- launchers (defined in the .cu files) -------------------------------------------
 cudaError_t launch_append(const AppendParams& p, int grid_x, cudaStream_t s);
-cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStream_t s, int overlap = 0);
+cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStream_t s, int overlap = 0, int n_layers = 1);
 cudaError_t launch_regroup(const GatherParams& p, cudaStream_t s, int programmatic);
 cudaError_t launch_reset(int* len, int* pos, int L, int B, int ring, int seq, cudaStream_t s);
 cudaError_t decode_setup();

@@ -116,6 +116,20 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     if (p.gdc_wait == 2) asm volatile("griddepcontrol.wait;" ::: "memory");   // before anything is read
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+    // ---- which layer (a launch may cover several layers of a decode step: blockIdx.y) -----------
+    const int li = p.layer_ids ? p.layer_ids[blockIdx.y] : 0;
+    int* const len_p = p.len + (long long)li * p.st_len;
+    int* const pos_p = p.pos + (long long)li * p.st_pos;
+    const __nv_bfloat16* const q_p = p.q + (long long)li * p.st_q;
+    __nv_bfloat16* const out_p = p.out + (long long)li * p.st_q;
+    const __nv_bfloat16* const k_new_p = p.k_new ? p.k_new + (long long)li * p.st_kv : nullptr;
+    const __nv_bfloat16* const v_new_p = p.v_new ? p.v_new + (long long)li * p.st_kv : nullptr;
+    const int* const head_list_p = p.head_list + (long long)li * p.n_kv_total;
+    unsigned int* const counters_p = p.counters + (long long)li * p.st_cnt;
+    unsigned int* const seq_counters_p = p.seq_counters + (long long)li * p.st_cnt;
+    float* const part_o_p = p.part_o + (long long)li * p.st_part * kD;
+    float* const part_ml_p = p.part_ml + (long long)li * p.st_part * 2;
+
     // ---- which work item -----------------------------------------------------------
     const int item = blockIdx.x;
     int b = 0;
@@ -125,22 +139,23 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     const int split = local / p.Hg;
     const int nsplit = p.split_start[b + 1] - p.split_start[b];
 
-    const bool fused = p.k_new != nullptr;
-    const int len_old = p.len[b];
+    const bool fused = k_new_p != nullptr;
+    const int len_old = len_p[b];
+    const SeqDesc sd = p.layer_ids ? p.desc_table[(long long)li * p.B + b] : p.sd[b];
     const int len = len_old + (fused ? 1 : 0);
     const int n = (p.kind == ZZ_KIND_RETRIEVAL) ? len : min(len, p.ring);
-    const long long slots_per_head = (p.kind == ZZ_KIND_RETRIEVAL) ? p.sd[b].cap : p.ring;
-    __nv_bfloat16* kbase = p.arena + p.sd[b].k_off[p.kind] + (long long)hg * slots_per_head * kD;
-    __nv_bfloat16* vbase = p.arena + p.sd[b].v_off[p.kind] + (long long)hg * slots_per_head * kD;
+    const long long slots_per_head = (p.kind == ZZ_KIND_RETRIEVAL) ? sd.cap : p.ring;
+    __nv_bfloat16* kbase = p.arena + sd.k_off[p.kind] + (long long)hg * slots_per_head * kD;
+    __nv_bfloat16* vbase = p.arena + sd.v_off[p.kind] + (long long)hg * slots_per_head * kD;
     int new_slot = -1;
     const __nv_bfloat16* knew = nullptr;
     const __nv_bfloat16* vnew = nullptr;
     if (fused) {
         const int t = len_old;
         new_slot = (p.kind == ZZ_KIND_RETRIEVAL || t < p.S) ? t : p.S + ((t - p.S) % p.W);
-        const long long src = ((long long)b * p.n_kv_total + p.head_list[p.kv_head0 + hg]) * kD;
-        knew = p.k_new + src;
-        vnew = p.v_new + src;
+        const long long src = ((long long)b * p.n_kv_total + head_list_p[p.kv_head0 + hg]) * kD;
+        knew = k_new_p + src;
+        vnew = v_new_p + src;
     }
 
     const int s0 = min(split * p.chunk[b], n);
@@ -154,12 +169,12 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
         const __nv_bfloat16* src = (lane < 16 ? knew : vnew) + c * 8;
         __nv_bfloat16* dst = (lane < 16 ? kbase : vbase) + (long long)new_slot * kD + c * 8;
         *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
-        if (p.kind == ZZ_KIND_STREAMING && hg == 0 && lane == 0) p.pos[(long long)b * p.ring + new_slot] = len_old;
+        if (p.kind == ZZ_KIND_STREAMING && hg == 0 && lane == 0) pos_p[(long long)b * p.ring + new_slot] = len_old;
     }
 
     // ---- query fragments: rows = the G heads of this KV head ---------------------------
     const int G = p.G;
-    const __nv_bfloat16* qb = p.q + ((long long)b * p.q_tok_stride) + (long long)(p.q_head0 + hg * G) * kD;
+    const __nv_bfloat16* qb = q_p + ((long long)b * p.q_tok_stride) + (long long)(p.q_head0 + hg * G) * kD;
     uint32_t qa[8][4];
 #pragma unroll
     for (int kk = 0; kk < 8; ++kk) {
@@ -310,7 +325,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     __syncthreads();
 
     const long long pair = (long long)b * p.Hg + hg;
-    __nv_bfloat16* outb = p.out + ((long long)b * p.q_tok_stride) + (long long)(p.q_head0 + hg * G) * kD;
+    __nv_bfloat16* outb = out_p + ((long long)b * p.q_tok_stride) + (long long)(p.q_head0 + hg * G) * kD;
     for (int idx = threadIdx.x; idx < G * kD; idx += kWarps * 32) {
         const int row = idx >> 7, d = idx & 127;
         float M = -INFINITY;
@@ -328,10 +343,10 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
             outb[row * kD + d] = __float2bfloat16_rn(acc / L);
         } else {
             const long long po = (long long)item * G + row;   // partials are indexed by work item
-            p.part_o[po * kD + d] = acc;
+            part_o_p[po * kD + d] = acc;
             if (d == 0) {
-                p.part_ml[po * 2 + 0] = M;
-                p.part_ml[po * 2 + 1] = L;
+                part_ml_p[po * 2 + 0] = M;
+                part_ml_p[po * 2 + 1] = L;
             }
         }
     }
@@ -341,10 +356,10 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
         __syncthreads();
         if (threadIdx.x == 0) {
             const unsigned int all = (unsigned int)(nsplit * p.Hg);
-            const unsigned int prev = atomicAdd(p.seq_counters + b, 1u);
+            const unsigned int prev = atomicAdd(seq_counters_p + b, 1u);
             if (prev == all - 1) {
-                p.len[b] = len_old + 1;
-                p.seq_counters[b] = 0u;
+                len_p[b] = len_old + 1;
+                seq_counters_p[b] = 0u;
             }
         }
     }
@@ -354,7 +369,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
-        const unsigned int prev = atomicAdd(p.counters + pair, 1u);
+        const unsigned int prev = atomicAdd(counters_p + pair, 1u);
         s_is_last = (prev == (unsigned int)(nsplit - 1));
     }
     __syncthreads();
@@ -371,7 +386,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
         const bool row_ok = row < G;
         // split s of this (sequence, head) is work item item0 + s * Hg
         const long long item0 = (long long)p.split_start[b] * p.Hg + hg;
-        const float* pbase = p.part_o + (item0 * G + (row_ok ? row : 0)) * kD + lane * 4;
+        const float* pbase = part_o_p + (item0 * G + (row_ok ? row : 0)) * kD + lane * 4;
         const long long sstride = (long long)p.Hg * G * kD;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int sb = 0; sb < nsplit; sb += kRound) {
@@ -385,7 +400,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
                     const int s = i / kWarps, r = row0 + i % kWarps;
                     if (r < G) {
                         const long long po = (item0 + (long long)s * p.Hg) * G + r;
-                        const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + po * 2));
+                        const float2 ml = __ldcg(reinterpret_cast<const float2*>(part_ml_p + po * 2));
                         sm_m[r * kMaxSplitsSmem + s] = ml.x;
                         sm_f[r * kMaxSplitsSmem + s] = ml.y;
                     }
@@ -426,7 +441,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
         }
         __syncthreads();
     }
-    if (threadIdx.x == 0) p.counters[pair] = 0u;
+    if (threadIdx.x == 0) counters_p[pair] = 0u;
 }
 
 }  // namespace
@@ -453,11 +468,11 @@ cudaError_t decode_setup() {
 // shares nothing at all with the previous one and does not wait for it.  overlap == 3: the kernel
 // waits for the previous launch at entry, before it reads anything (always safe; only the launch
 // latency overlaps).
-cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStream_t s, int overlap) {
+cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStream_t s, int overlap, int n_layers) {
     if (n_items <= 0) return cudaSuccess;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3(n_items);
+    cfg.gridDim = dim3(n_items, n_layers > 0 ? n_layers : 1);
     cfg.blockDim = dim3(warps * 32);
     cfg.dynamicSmemBytes = warps * kWarpSmem;
     cfg.stream = s;
