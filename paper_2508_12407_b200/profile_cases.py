@@ -5,7 +5,8 @@
 Each case holds well under a few GB on the device and its inputs exceed the 126 MB L2, so a
 capture of one to three launches ends by itself and its DRAM counters are meaningful.
 Cases: decode_r (retrieval decode), decode_s (streaming decode), prefill_r, prefill_s,
-append (decode-time append), mixed (mixed-head decode layer).
+append (decode-time append), mixed (mixed-head decode layer), decode_all (whole-stack decode step:
+layers alternate retrieval / streaming, one grid per kind, as the benchmark launches it).
 """
 from __future__ import annotations
 
@@ -20,7 +21,7 @@ from . import binding, build
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--case", required=True,
-                    choices=["decode_r", "decode_s", "prefill_r", "prefill_s", "append", "mixed"])
+                    choices=["decode_r", "decode_s", "decode_all", "prefill_r", "prefill_s", "append", "mixed"])
     ap.add_argument("--n", type=int, default=32768, help="context length (decode) or chunk length (prefill)")
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--layers", type=int, default=2)
@@ -39,10 +40,13 @@ def main():
         return torch.randn(*shape, device=dev, generator=g, dtype=torch.float32).to(torch.bfloat16)
 
     kind = 1 if args.case in ("decode_r", "prefill_r", "append") else 0
+    kinds = [kind] * L
+    if args.case == "decode_all":
+        kinds = [1 - (l & 1) for l in range(L)]
     kvk = None
     if args.case == "mixed":
         kvk = np.tile(np.array([1, 0, 1, 0, 0, 1, 1, 0], dtype=np.uint8), (L, 1))
-    cache = binding.ZigzagCache(L, B, Hq, Hkv, S, W, [kind] * L, [N + 64] * B, max(B * N, B),
+    cache = binding.ZigzagCache(L, B, Hq, Hkv, S, W, kinds, [N + 64] * B, max(B * N, B),
                                 kvhead_is_retrieval=kvk)
     if args.case in ("prefill_r", "prefill_s"):
         q, k, v = randn(B * N, Hq, D), randn(B * N, Hkv, D), randn(B * N, Hkv, D)
@@ -60,6 +64,12 @@ def main():
                 done += c
         q, k, v = randn(B, Hq, D), randn(B, Hkv, D), randn(B, Hkv, D)
         out = torch.empty_like(q)
+        if args.case == "decode_all":
+            qa, ka, va = randn(L, B, Hq, D), randn(L, B, Hkv, D), randn(L, B, Hkv, D)
+            oa = torch.empty_like(qa)
+            for _ in range(args.reps):
+                cache.decode_step_all(qa, ka, va, oa)
+            args.reps = 0
         for _ in range(args.reps):
             for l in range(L):
                 if args.case == "append":
