@@ -86,19 +86,6 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Non-blocking probe of a phase (try_wait may suspend the thread for a while when the phase is
-// still open; a probe must not).
-__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
 // Bounded wait.  Returns false (after flagging the error) if the phase never completed.
 // The first probe is inlined: a wait on a phase that has already completed costs one
 // try_wait, and only a real wait enters the polling loop.
@@ -592,8 +579,16 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                 // tile_masked: some entry of this 128 x 128 tile may be invisible (uniform over the
                 // CTA); vis[w] bit i: column 32 w + i is visible to this thread's row
                 bool tile_masked = true;
-                if (p.kind == ZZ_KIND_RETRIEVAL)
+                if (p.kind == ZZ_KIND_RETRIEVAL) {
                     tile_masked = is_chunk ? (start + 127 > r0) : (plan.n_occ - start < 128);
+                } else if (is_chunk) {
+                    // a chunk tile of a streaming layer is fully visible to all 128 rows if it lies
+                    // below the diagonal and either inside every row's window or among the sinks
+                    const bool below = start + 127 <= r0;
+                    const bool in_window = start >= r0 + 127 - p.W + 1;
+                    const bool all_sinks = start + 127 < p.S - P;
+                    tile_masked = !(below && (in_window || all_sinks));
+                }
                 if (tile_masked) {
                     uint32_t vis[4];
                     if (p.kind == ZZ_KIND_RETRIEVAL) {
