@@ -707,16 +707,21 @@ int zz_decode_step_all(zz_cache_t* c, const void* d_q, const void* d_k, const vo
         const __nv_bfloat16* k = static_cast<const __nv_bfloat16*>(d_k);
         const __nv_bfloat16* v = static_cast<const __nv_bfloat16*>(d_v);
         __nv_bfloat16* out = static_cast<__nv_bfloat16*>(d_out);
+        // The short streaming grid goes first as an ordinary launch; the retrieval grid follows as a
+        // programmatic launch (it starts while the streaming CTAs run) whose CTAs execute
+        // griddepcontrol.wait after their main loop, long after the streaming grid has finished.  So
+        // the retrieval grid completes after the streaming grid, and whatever follows in the stream
+        // only has to wait for the last launch.
         int r = ZZ_OK;
         bool first = true;
-        if (c->n_excl_R > 0) {
-            r = launch_decode_group(c, c->layer_ids[0], ZZ_KIND_RETRIEVAL, q, out, 0, st, k, v, 1, 0, c->d_layer_ids(),
-                                    c->n_excl_R);
+        if (c->n_excl_S > 0) {
+            r = launch_decode_group(c, c->layer_ids[c->n_excl_R], ZZ_KIND_STREAMING, q, out, 0, st, k, v, 1, 0,
+                                    c->d_layer_ids() + c->n_excl_R, c->n_excl_S);
             first = false;
         }
-        if (r == ZZ_OK && c->n_excl_S > 0)
-            r = launch_decode_group(c, c->layer_ids[c->n_excl_R], ZZ_KIND_STREAMING, q, out, 0, st, k, v, 1,
-                                    first ? 0 : 2, c->d_layer_ids() + c->n_excl_R, c->n_excl_S);
+        if (r == ZZ_OK && c->n_excl_R > 0)
+            r = launch_decode_group(c, c->layer_ids[0], ZZ_KIND_RETRIEVAL, q, out, 0, st, k, v, 1, first ? 0 : 1,
+                                    c->d_layer_ids(), c->n_excl_R);
         if (r != ZZ_OK) return r;
         for (size_t i = 0; i < c->len.size(); ++i) c->len[i] += 1;
         return ZZ_OK;
