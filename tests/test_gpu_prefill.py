@@ -129,6 +129,15 @@ def test_maximum_batch_packed_prefill():
     run_prefill(2, binding.ZZ_MAX_BATCH, 4, 2, 8, 24, [1, 0], plans, seed=65, n_decode=1)
 
 
+def test_odd_group_many_items_persistent_path():
+    # odd group size (the second tile of some head pairs is absent) with more work items than SMs,
+    # so the streaming layer runs persistent CTAs that meet both kinds of item; two chunks, so the
+    # second one also reads ring tiles
+    def rows(P, c):
+        return [0, 1, 127, 128, 129, 255, 256, 383, 384, c // 2, c - 130, c - 1]
+    run_prefill(2, 1, 3, 1, 100, 200, [0, 1], [[128 * 90 + 5, 128 * 80 + 77]], seed=81, sample_rows=rows)
+
+
 def test_decode_step_equals_prefill_row():
     # the last row of a prefill and a decode step at the same position agree within tolerance
     D, S, W, n = 128, 32, 64, 500
