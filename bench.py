@@ -137,10 +137,10 @@ def run_reference(args, w):
         return
     vals = []
     for _ in range(args.warmup):
-        oracle_sample(w, 1)
+        oracle_sample(w, 8)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        cb = oracle_sample(w, 2)
+        cb = oracle_sample(w, 64)
         vals.append(cb["value"])
     ms = (time.perf_counter() - t0) * 1e3 / max(1, args.steps)
     v = float(np.mean(vals))
@@ -429,7 +429,7 @@ def run_ours(args, w):
     # ---- CPU oracle baseline (rank 0, single GPU only) -----------------------------------------
     if rank == 0 and world == 1 and not args.no_cpu:
         try:
-            line["cpu_baseline"] = oracle_sample(w, 2)
+            line["cpu_baseline"] = oracle_sample(w, 256)     # ~10 s of oracle work on the host cores
         except Exception as e:  # the oracle is optional for the timing itself
             line["cpu_baseline"] = {"error": str(e)}
     cache.close()
