@@ -109,6 +109,9 @@ class ClockSampler:
 
 # --------------------------------------------------------------------------- oracle (CPU) leg
 
+_ORACLE_INPUTS = {}
+
+
 def oracle_sample(w: inputs.Workload, n_rows: int = 2):
     """Times the fp64 oracle on decode rows of one retrieval and one streaming layer at the
     workload's context length and extrapolates to one token over the whole stack."""
@@ -120,7 +123,10 @@ def oracle_sample(w: inputs.Workload, n_rows: int = 2):
     t_rows = np.arange(N - n_rows, N)
     secs = {}
     for name, layer, kind in (("retrieval", lR, 1), ("streaming", lS, 0)):
-        q, k, v = inputs.qkv_bf16(w, layer, 0, 0, N)
+        key = (w.name, layer, N)
+        if key not in _ORACLE_INPUTS:          # the seeded inputs are drawn once, outside the timing
+            _ORACLE_INPUTS[key] = inputs.qkv_bf16(w, layer, 0, 0, N)
+        q, k, v = _ORACLE_INPUTS[key]
         t0 = time.perf_counter()
         oracle.attn_rows(np.ascontiguousarray(q[t_rows]), t_rows, k, v, [kind] * w.n_kv_heads, w.sink, w.recent, w.scale)
         secs[name] = (time.perf_counter() - t0) / n_rows
