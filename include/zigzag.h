@@ -114,7 +114,8 @@ int zz_cache_len(const zz_cache_t* cache, int layer, int seq, int32_t* len);
  * layers hold equally long sequences; otherwise as 2); 2: one launch per layer, programmatic
  * dependent launch and no wait between layers -- they share no scratch, so a layer's kernel fills
  * the SMs the previous one leaves idle; 1: the same, but each kernel waits for the previous one
- * before it merges; 0: plain stream order). */
+ * before it merges; 0: plain stream order); "decode_multi_waves" (default 8: a grid over n layers
+ * cuts every layer into about 2 * SMs * value / n work items instead of 2 * SMs). */
 int zz_tune(zz_cache_t* cache, const char* key, int value);
 
 /* KV append with sink + recent eviction (paper: Introduction -- the KV cache grows with

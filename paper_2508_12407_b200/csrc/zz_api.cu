@@ -132,6 +132,7 @@ struct zz_cache {
     int decode_min_chunk;
     int decode_short_tokens;
     int decode_overlap;
+    int decode_multi_waves;
     bool last_nowait;   // the last launch did not wait for its predecessor: the next one must be an ordinary launch
     bool has_mixed;
     alignas(64) CUtensorMap tmap_arena;
@@ -240,7 +241,7 @@ bool bad_layer(const zz_cache* c, int layer) { return !c || layer < 0 || layer >
 // Split plan of one decode launch.  Short stores: 8-warp CTAs (one per SM) that each take up to
 // 384 tokens, so a warp's chain is at most three dependent steps.  Long stores: 4-warp CTAs
 // (two per SM), all work items in one wave, every sequence cut into equal splits.
-void plan_splits(const zz_cache* c, const int* n, int Hg, int* warps, int* chunk, int* split_start) {
+void plan_splits(const zz_cache* c, const int* n, int Hg, int* warps, int* chunk, int* split_start, int n_multi = 1) {
     long long total = 0;
     for (int b = 0; b < c->B; ++b) total += n[b];
     split_start[0] = 0;
@@ -255,7 +256,16 @@ void plan_splits(const zz_cache* c, const int* n, int Hg, int* warps, int* chunk
         return;
     }
     *warps = 4;
-    const int slots = 2 * c->num_sms < kMaxSlots ? 2 * c->num_sms : kMaxSlots;
+    int slots = 2 * c->num_sms < kMaxSlots ? 2 * c->num_sms : kMaxSlots;
+    // a grid over several layers fills the GPU with all of them together: each layer is cut into
+    // fewer, longer items (decode_multi_waves waves of CTAs over the whole grid), which spends less
+    // on per-CTA ramp-up, merge and partials
+    if (n_multi > 1) {
+        int s = (int)(((long long)slots * c->decode_multi_waves + n_multi - 1) / n_multi);
+        const int floor_items = 4 * c->B * Hg;        // keep several splits per sequence for ragged batches
+        if (s < floor_items) s = floor_items;
+        if (s < slots) slots = s;
+    }
     long long per = (total * Hg + slots - 1) / slots;   // tokens per work item if all were equal
     if (per < c->decode_min_chunk) per = c->decode_min_chunk;
     for (;;) {
@@ -321,7 +331,7 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
         n[b] = (kind == ZZ_KIND_RETRIEVAL) ? len : (len < c->ring ? len : c->ring);
     }
     int warps = 4;
-    plan_splits(c, n, Hg, &warps, p.chunk, p.split_start);
+    plan_splits(c, n, Hg, &warps, p.chunk, p.split_start, d_layer_ids ? n_multi : 1);
     const int items = p.split_start[c->B] * Hg;
     const int pk = (kind == ZZ_KIND_RETRIEVAL) ? zz::kProfDecodeR : zz::kProfDecodeS;
     zz::prof_begin(pk, st);
@@ -466,6 +476,7 @@ int zz_cache_create(const zz_config_t* cfg, void* d_arena, size_t arena_bytes, v
     c->decode_short_tokens = 384;
     c->decode_overlap = 3;
     c->last_nowait = false;
+    c->decode_multi_waves = 8;
     compute_layout(cfg, &c->lay, &c->desc);
     if (arena_bytes < c->lay.arena_bytes || workspace_bytes < c->lay.work_bytes) {
         delete c;
@@ -556,6 +567,11 @@ int zz_tune(zz_cache_t* c, const char* key, int value) {
     if (!strcmp(key, "decode_min_chunk")) {
         if (value < 16 || value % 16) return ZZ_ERR_INVALID_ARG;
         c->decode_min_chunk = value;
+        return ZZ_OK;
+    }
+    if (!strcmp(key, "decode_multi_waves")) {
+        if (value < 1 || value > 64) return ZZ_ERR_INVALID_ARG;
+        c->decode_multi_waves = value;
         return ZZ_OK;
     }
     if (!strcmp(key, "decode_overlap")) {
