@@ -328,7 +328,8 @@ def run_ours(args, w):
         heads_R = Hkv if kvk is None else (w.mixed_retrieval_kv_heads or Hkv // 2)
         bytes_launch = float((2 * heads_R * avg_n * D * 2).sum()) + B * heads_R * (Hq // Hkv) * D * 2 * 2
         # with the default launch mode one grid covers all retrieval layers of a step
-        layers_per_launch = nR_layers if (kvk is None and args.decode_overlap in (-1, 3)) else 1
+        # (mixed arm: one grid covers the retrieval heads of every layer)
+        layers_per_launch = (nR_layers if kvk is None else L) if args.decode_overlap in (-1, 3) else 1
         bytes_launch *= layers_per_launch
         roofs["decode_retrieval"] = roof("decode_kernel (retrieval layers; a sampled launch, serialised against its neighbours)", "hbm",
                                          bytes_launch / (ms_dr / n_dr * 1e-3) / 1e9, p["hbm_gbs"], "GB/s",
@@ -363,7 +364,8 @@ def run_ours(args, w):
         dec_bytes_step = fr * float((2 * Hkv * avg_n_all * D * 2).sum()) + fs * float(
             (2 * Hkv * np.minimum(avg_n_all, ring) * D * 2).sum()) + L * B * (2 * Hq * D * 2 + 4 * Hkv * D * 2)
         n_dec_launches = sum(m[3] for m in all_marks)
-        roofs["decode_step"] = roof("decode_kernel (all launches of the decode phase: per step one grid over the retrieval layers, one over the streaming layers)",
+        roofs["decode_step"] = roof("decode_kernel (all launches of the decode phase: per step one grid over the retrieval layers"
+                                    " or heads, one over the streaming ones; the mixed arm adds two regrouping copies)",
                                     "hbm", dec_bytes_step * steps_dec * K / (dec_ms * 1e-3) / 1e9, p["hbm_gbs"],
                                     "GB/s", "decode_step")
         roofs["decode_step"]["us_per_launch"] = dec_ms * 1e3 / max(1, n_dec_launches)

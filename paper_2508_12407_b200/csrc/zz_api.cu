@@ -63,7 +63,7 @@ size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 struct Layout {
     // workspace sections (byte offsets)
     size_t off_status, off_len, off_pos, off_desc, off_heads, off_counters, off_part_ml, off_part_o,
-        off_qc, off_oc, off_layer_ids, work_bytes;
+        off_qc, off_oc, off_dqc, off_doc, off_layer_ids, work_bytes;
     size_t arena_bytes, counters_per_layer, items_per_layer;
 };
 
@@ -123,8 +123,9 @@ struct zz_cache {
     std::vector<int> cap;             // [B]
     std::vector<int> len;             // [L*B] host mirror
     std::vector<SeqDesc> desc;        // [L*B]
-    std::vector<int> layer_ids;       // exclusive retrieval layers (ascending), then exclusive streaming layers
-    int n_excl_R, n_excl_S;
+    std::vector<int> layer_ids;       // exclusive retrieval layers (ascending), exclusive streaming, mixed
+    int n_excl_R, n_excl_S, n_mixed;
+    bool mixed_same_nR;               // every mixed layer has the same number of retrieval heads
     Layout lay;
     unsigned char* arena;
     unsigned char* work;
@@ -156,6 +157,9 @@ struct zz_cache {
     }
     __nv_bfloat16* d_qc() const { return reinterpret_cast<__nv_bfloat16*>(work + lay.off_qc); }
     __nv_bfloat16* d_oc() const { return reinterpret_cast<__nv_bfloat16*>(work + lay.off_oc); }
+    // compact-order q and out of a decode step over all layers: [L][B][Hq][128]
+    __nv_bfloat16* d_dqc() const { return reinterpret_cast<__nv_bfloat16*>(work + lay.off_dqc); }
+    __nv_bfloat16* d_doc() const { return reinterpret_cast<__nv_bfloat16*>(work + lay.off_doc); }
     __nv_bfloat16* d_arena() const { return reinterpret_cast<__nv_bfloat16*>(arena); }
     bool mixed(int l) const { return nR[l] > 0 && nR[l] < Hkv; }
 };
@@ -233,6 +237,10 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
     if (has_mixed) w += align_up((size_t)c->max_new_tokens * Hq * kD * 2);
     lay->off_oc = w;
     if (has_mixed) w += align_up((size_t)c->max_new_tokens * Hq * kD * 2);
+    lay->off_dqc = w;
+    if (has_mixed) w += align_up((size_t)L * B * Hq * kD * 2);
+    lay->off_doc = w;
+    if (has_mixed) w += align_up((size_t)L * B * Hq * kD * 2);
     lay->work_bytes = w;
 }
 
@@ -369,11 +377,19 @@ int regroup(zz_cache* c, int layer, const __nv_bfloat16* src, __nv_bfloat16* dst
     zz::GatherParams g;
     g.src = src;
     g.dst = dst;
-    g.head_list = c->d_heads(layer);
+    g.head_list = c->d_heads(layer < 0 ? 0 : layer);
     g.Hkv = c->Hkv;
     g.G = c->G;
     g.tokens = tokens;
     g.to_compact = to_compact;
+    g.layer_ids = nullptr;
+    g.toks_per_layer = 0;
+    if (layer < 0) {
+        // every mixed layer of a decode step at once (tokens = n_mixed * B)
+        g.head_list = c->d_heads(0);
+        g.layer_ids = c->d_layer_ids() + c->n_excl_R + c->n_excl_S;
+        g.toks_per_layer = c->B;
+    }
     zz::prof_begin(zz::kProfRegroup, st);
     const cudaError_t e = zz::launch_regroup(g, st, c->last_nowait ? 0 : 1);
     c->last_nowait = false;
@@ -507,7 +523,14 @@ int zz_cache_create(const zz_config_t* cfg, void* d_arena, size_t arena_bytes, v
         if (c->nR[l] == c->Hkv) { c->layer_ids.push_back(l); ++c->n_excl_R; }
     for (int l = 0; l < c->L; ++l)
         if (c->nR[l] == 0) { c->layer_ids.push_back(l); ++c->n_excl_S; }
-    c->layer_ids.resize(c->L, 0);
+    c->n_mixed = 0;
+    c->mixed_same_nR = true;
+    for (int l = 0; l < c->L; ++l)
+        if (c->mixed(l)) {
+            if (c->n_mixed > 0 && c->nR[l] != c->nR[c->layer_ids.back()]) c->mixed_same_nR = false;
+            c->layer_ids.push_back(l);
+            ++c->n_mixed;
+        }
     c->cap.assign(cfg->capacity, cfg->capacity + c->B);
     c->len.assign((size_t)c->L * c->B, 0);
 
@@ -707,12 +730,14 @@ int zz_decode_step_all(zz_cache_t* c, const void* d_q, const void* d_k, const vo
     for (int l = 0; l < c->L; ++l)
         for (int b = 0; b < c->B; ++b)
             if (c->nR[l] > 0 && c->len[(size_t)l * c->B + b] + 1 > c->cap[b]) return ZZ_ERR_CAPACITY;
-    // All layers exclusive and of equal lengths: one launch for the retrieval layers and one for the
-    // streaming layers (blockIdx.y = layer).  The layers are independent (own stores, lengths,
-    // scratch and output slice; q/k/v of all layers are inputs of the call), so a launch over many
-    // layers only removes launch boundaries: no ramp-up and tail per layer, and the ~3 us per launch
-    // that a streaming layer's few CTAs cannot fill.
-    bool same_len = !c->has_mixed && c->decode_overlap == 3;
+    // Equal lengths in every layer: one launch per kind of work instead of one (or four) per layer
+    // (blockIdx.y = layer).  The layers are independent (own stores, lengths, scratch and output
+    // slice; q/k/v of all layers are inputs of the call), so a launch over many layers only removes
+    // launch boundaries: no ramp-up and tail per layer, and the ~3 us per launch that a streaming
+    // layer's few CTAs cannot fill.  Mixed layers join when they all have the same number of
+    // retrieval heads (one split plan serves them all): one regrouping launch before and one after,
+    // and their two passes ride in grids of their own.
+    bool same_len = c->decode_overlap == 3 && (c->n_mixed == 0 || c->mixed_same_nR);
     for (int l = 1; l < c->L && same_len; ++l)
         for (int b = 0; b < c->B; ++b)
             if (c->len[(size_t)l * c->B + b] != c->len[b]) same_len = false;
@@ -723,21 +748,38 @@ int zz_decode_step_all(zz_cache_t* c, const void* d_q, const void* d_k, const vo
         const __nv_bfloat16* k = static_cast<const __nv_bfloat16*>(d_k);
         const __nv_bfloat16* v = static_cast<const __nv_bfloat16*>(d_v);
         __nv_bfloat16* out = static_cast<__nv_bfloat16*>(d_out);
-        // The short streaming grid goes first as an ordinary launch; the retrieval grid follows as a
-        // programmatic launch (it starts while the streaming CTAs run) whose CTAs execute
-        // griddepcontrol.wait after their main loop, long after the streaming grid has finished.  So
-        // the retrieval grid completes after the streaming grid, and whatever follows in the stream
-        // only has to wait for the last launch.
+        // Order: [regroup q of the mixed layers], the short streaming grids, then the retrieval
+        // grids, [regroup the mixed layers' outputs].  The first decode grid is an ordinary launch
+        // (it starts after the regrouping copy has completed).  Every later grid is a programmatic
+        // launch: it starts while its predecessor's CTAs run and executes griddepcontrol.wait after
+        // its main loop, before it touches the split scratch, the output or the lengths.  A grid
+        // therefore completes only after its predecessor has, so the chain completes in order, the
+        // two passes of a mixed layer never share scratch at the same time, and whatever follows in
+        // the stream only has to wait for the last launch.
+        const int* ids = c->d_layer_ids();
+        const int oS = c->n_excl_R, oM = c->n_excl_R + c->n_excl_S;
         int r = ZZ_OK;
         bool first = true;
-        if (c->n_excl_S > 0) {
-            r = launch_decode_group(c, c->layer_ids[c->n_excl_R], ZZ_KIND_STREAMING, q, out, 0, st, k, v, 1, 0,
-                                    c->d_layer_ids() + c->n_excl_R, c->n_excl_S);
+        if (c->n_mixed > 0) r = regroup(c, -1, q, c->d_dqc(), (long long)c->n_mixed * c->B, 1, st);
+        if (r == ZZ_OK && c->n_excl_S > 0) {
+            r = launch_decode_group(c, c->layer_ids[oS], ZZ_KIND_STREAMING, q, out, 0, st, k, v, 1, first ? 0 : 1,
+                                    ids + oS, c->n_excl_S);
             first = false;
         }
+        if (r == ZZ_OK && c->n_mixed > 0) {
+            const int lm = c->layer_ids[oM];
+            r = launch_decode_group(c, lm, ZZ_KIND_STREAMING, c->d_dqc(), c->d_doc(), c->nR[lm] * c->G, st, k, v, 0,
+                                    first ? 0 : 1, ids + oM, c->n_mixed);
+            first = false;
+            // the retrieval pass is the layer's last: it publishes the new lengths
+            if (r == ZZ_OK)
+                r = launch_decode_group(c, lm, ZZ_KIND_RETRIEVAL, c->d_dqc(), c->d_doc(), 0, st, k, v, 1, 1, ids + oM,
+                                        c->n_mixed);
+        }
         if (r == ZZ_OK && c->n_excl_R > 0)
-            r = launch_decode_group(c, c->layer_ids[0], ZZ_KIND_RETRIEVAL, q, out, 0, st, k, v, 1, first ? 0 : 1,
-                                    c->d_layer_ids(), c->n_excl_R);
+            r = launch_decode_group(c, c->layer_ids[0], ZZ_KIND_RETRIEVAL, q, out, 0, st, k, v, 1, first ? 0 : 1, ids,
+                                    c->n_excl_R);
+        if (r == ZZ_OK && c->n_mixed > 0) r = regroup(c, -1, c->d_doc(), out, (long long)c->n_mixed * c->B, 0, st);
         if (r != ZZ_OK) return r;
         for (size_t i = 0; i < c->len.size(); ++i) c->len[i] += 1;
         return ZZ_OK;

@@ -115,8 +115,14 @@ __global__ void __launch_bounds__(256) regroup_kernel(const GatherParams p) {
         const int g = (int)(r % p.G);
         r /= p.G;
         const int c = (int)(r % p.Hkv);   // compact KV-head index
-        const long long tok = r / p.Hkv;
-        const int h = p.head_list[c];     // model KV-head index
+        long long tok = r / p.Hkv;
+        const int* hl = p.head_list;
+        if (p.layer_ids) {
+            const int layer = p.layer_ids[tok / p.toks_per_layer];
+            tok = (long long)layer * p.toks_per_layer + tok % p.toks_per_layer;
+            hl += (long long)layer * p.Hkv;
+        }
+        const int h = hl[c];              // model KV-head index
         const long long compact = ((tok * p.Hkv + c) * p.G + g) * kD + piece * 8;
         const long long model = ((tok * p.Hkv + h) * p.G + g) * kD + piece * 8;
         if (p.to_compact)

@@ -85,6 +85,10 @@ struct GatherParams {
     int Hkv, G;
     long long tokens;
     int to_compact;          // 1: model order -> compact (gather); 0: compact -> model order (scatter)
+    // several layers in one launch (decode step): token t belongs to layer layer_ids[t / toks_per_layer];
+    // src, dst and head_list are then the layer-0 pointers, each layer `toks_per_layer` tokens further
+    const int* layer_ids;    // nullptr: one layer
+    int toks_per_layer;
 };
 
 struct PrefillParams {

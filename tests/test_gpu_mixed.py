@@ -59,3 +59,63 @@ def test_mixed_equals_exclusive_per_head():
         src = "R" if kinds[h // G] else "S"
         assert np.array_equal(outs["M"][0][:, h], outs[src][0][:, h])
         assert np.array_equal(outs["M"][1][:, h], outs[src][1][:, h])
+
+
+@pytest.mark.parametrize("same_nr", [True, False])
+def test_whole_stack_step_with_mixed_layers(same_nr):
+    """A decode step over a stack of mixed and exclusive layers: the launches batched over layers
+    (mixed layers with equal retrieval-head counts) give the bits of the layer-by-layer path, the
+    cache contents agree bit for bit, and the last step matches the oracle.  With unequal counts
+    the batched path must decline and the layer-by-layer path runs."""
+    import torch
+    from test_gpu_append_decode import make
+    from zz_testlib import OracleSeq, assert_close
+    D, B, Hq, Hkv, S, W = 128, 2, 8, 4, 16, 48
+    kvk = np.array([[1, 0, 0, 1], [1, 1, 1, 1], [0, 1, 1, 0], [0, 0, 0, 0],
+                    [1, 1, 0, 0] if same_nr else [1, 1, 1, 0]], dtype=np.uint8)
+    L = len(kvk)
+    lens = [5000, 2300]
+    steps = 6
+    w = inputs.Workload("t", L, B, Hq, Hkv, D, S, W, 1, 0, 0, steps, seed=777)
+    hist = [[inputs.qkv_bf16(w, l, b, 0, lens[b]) for b in range(B)] for l in range(L)]
+    dec = [[[inputs.qkv_bf16(w, l, b, lens[b] + i, 1) for b in range(B)] for l in range(L)] for i in range(steps)]
+    results, stores = {}, {}
+    for mode in (0, 3):
+        cache = make(L, B, Hq, Hkv, S, W, [0] * L, [n + steps + 4 for n in lens], kvk=kvk, max_new=8192)
+        cache.tune("decode_overlap", mode)
+        for l in range(L):
+            k = np.concatenate([hist[l][b][1] for b in range(B)])
+            v = np.concatenate([hist[l][b][2] for b in range(B)])
+            cache.kv_append(l, to_dev(k), to_dev(v), lens)
+        outs = []
+        for i in range(steps):
+            q = np.stack([np.concatenate([dec[i][l][b][0] for b in range(B)]) for l in range(L)])
+            k = np.stack([np.concatenate([dec[i][l][b][1] for b in range(B)]) for l in range(L)])
+            v = np.stack([np.concatenate([dec[i][l][b][2] for b in range(B)]) for l in range(L)])
+            dq, dk, dv = to_dev(q), to_dev(k), to_dev(v)
+            out = torch.zeros_like(dq)
+            cache.decode_step_all(dq, dk, dv, out)
+            outs.append(to_bits(out))
+        torch.cuda.synchronize()
+        assert cache.last_status() == 0
+        results[mode] = np.stack(outs)
+        for l in range(L):
+            for b in range(B):
+                assert cache.len(l, b) == lens[b] + steps
+        stores[mode] = [cache.export(l, b, kind) for l in range(L) for b in range(B)
+                        for kind in (binding.KIND_RETRIEVAL, binding.KIND_STREAMING)
+                        if (kvk[l] == (kind == binding.KIND_RETRIEVAL)).any()]
+        cache.close()
+    assert np.array_equal(results[0], results[3])
+    for a, b_ in zip(stores[0], stores[3]):
+        for x, y in zip(a, b_):
+            assert np.array_equal(np.asarray(x), np.asarray(y))
+    scale = 1 / np.sqrt(D)
+    for l in range(L):
+        for b in range(B):
+            o = OracleSeq(Hkv, D, S, W, lens[b] + steps + 4, list(kvk[l]))
+            o.append(hist[l][b][1], hist[l][b][2])
+            for i in range(steps):
+                o.append(dec[i][l][b][1], dec[i][l][b][2])
+            want = o.rows(dec[steps - 1][l][b][0], [lens[b] + steps - 1], scale=scale)
+            assert_close(results[3][steps - 1, l, b:b + 1], want, f"layer {l} seq {b}")
