@@ -310,7 +310,8 @@ def run_ours(args, w):
     # decode bytes per step: K and V of the visible tokens + q + o + the appended rows (read + write)
     base_len = lens.astype(np.float64) if not C else np.full(B, float(w.prefill_len))
     p = peaks()
-    traffic = ncu_traffic()
+    # the committed DRAM counters are those of the cfg2 launches: other workloads report none
+    traffic = ncu_traffic() if (w.name == "cfg2" and not args.mixed and args.decode_overlap in (-1, 3)) else {}
 
     def roof(kind_name, bound, achieved, peak, unit, traffic_key):
         return {"kernel": kind_name, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
