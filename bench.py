@@ -193,8 +193,13 @@ def run_ours(args, w):
     # steps of every warm-up and timed step; prefilled workloads start each step from a reset
     rounds = 1 if C else (args.steps + args.warmup + 2)
     cap = [int(n) + rounds * steps_dec + 8 for n in lens]
+    pool_pages = 0
+    if args.paged:
+        # retrieval stores in 128-token pages: a pool of exactly the pages the capacities need
+        heads_R = int(kvk.sum()) if kvk is not None else int(np.sum(kinds)) * Hkv
+        pool_pages = heads_R * sum((c + 127) // 128 for c in cap)
     cache = binding.ZigzagCache(L, B, Hq, Hkv, w.sink, w.recent, kinds, cap, max(B, B * C), kvhead_is_retrieval=kvk,
-                                device=f"cuda:{local}")
+                                device=f"cuda:{local}", pool_pages=pool_pages)
 
     if args.decode_overlap >= 0:
         cache.tune("decode_overlap", args.decode_overlap)
@@ -311,7 +316,8 @@ def run_ours(args, w):
     base_len = lens.astype(np.float64) if not C else np.full(B, float(w.prefill_len))
     p = peaks()
     # the committed DRAM counters are those of the cfg2 launches: other workloads report none
-    traffic = ncu_traffic() if (w.name == "cfg2" and not args.mixed and args.decode_overlap in (-1, 3)) else {}
+    traffic = ncu_traffic() if (w.name == "cfg2" and not args.mixed and not args.paged
+                                and args.decode_overlap in (-1, 3)) else {}
 
     def roof(kind_name, bound, achieved, peak, unit, traffic_key):
         return {"kernel": kind_name, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
@@ -383,7 +389,7 @@ def run_ours(args, w):
     line = {"metric": METRIC, "value": us_per_token, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
             "ms_per_step": total_ms / K, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": w.name + ("+mixed" if args.mixed else ""), "layers": L, "batch": B,
+            "config": {"workload": w.name + ("+mixed" if args.mixed else "") + ("+paged" if args.paged else ""), "layers": L, "batch": B,
                        "q_heads": Hq, "kv_heads": Hkv, "head_dim": D, "sink": w.sink, "recent": w.recent,
                        "retrieval_layers": nR_layers, "prefill_len": w.prefill_len, "prefill_chunk": C,
                        "decode_steps": steps_dec, "decode_overlap": args.decode_overlap if args.decode_overlap >= 0 else 3,
@@ -455,6 +461,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--paged", action="store_true",
+                    help="retrieval stores in 128-token pages from a shared pool (a variant, not the default)")
     ap.add_argument("--decode-steps", type=int, default=-1, help="override the workload's decode steps")
     ap.add_argument("--mixed", action="store_true", help="mixed-head (two-pass) arm of the comparison")
     ap.add_argument("--share-inputs", action="store_true", help="one set of prefill tensors for all layers")

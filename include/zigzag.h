@@ -97,6 +97,22 @@ int zz_cache_query(const zz_config_t* cfg, size_t* arena_bytes, size_t* workspac
  * finished initialising).  *out is written only on success. */
 int zz_cache_create(const zz_config_t* cfg, void* d_arena, size_t arena_bytes, void* d_workspace,
                     size_t workspace_bytes, zz_cache_t** out);
+/* Paged retrieval stores (a variant the paper does not describe; the attention computed is the
+ * same).  The retrieval stores of all layers and sequences share one pool of `pool_pages` pages;
+ * a page holds 128 tokens of one KV head (its K rows, then its V rows: 64 KB).  A sequence takes
+ * pages as it grows (one per retrieval KV head of the layer per 128 tokens) and returns them in
+ * zz_cache_reset, so the pool may be smaller than the sum of the capacities; capacity[seq] stays
+ * the most tokens a sequence may hold (it sizes the page table).  Calls that add tokens
+ * (zz_kv_append, zz_decode_step, zz_decode_step_all, the *_host entries, zz_cache_import) return
+ * ZZ_ERR_CAPACITY, having launched and changed nothing, when the pool has too few free pages.
+ * Streaming rings are not paged.  Page bookkeeping lives on the host; its device-side table is
+ * written by small launches on the caller's stream, so one handle must be driven from one stream
+ * at a time.  Everything else behaves as with zz_cache_query / zz_cache_create. */
+int zz_cache_query_paged(const zz_config_t* cfg, int32_t pool_pages, size_t* arena_bytes, size_t* workspace_bytes);
+int zz_cache_create_paged(const zz_config_t* cfg, int32_t pool_pages, void* d_arena, size_t arena_bytes,
+                          void* d_workspace, size_t workspace_bytes, zz_cache_t** out);
+/* Pages of the pool and pages free now (both 0 for a cache with contiguous stores). */
+int zz_cache_pages(const zz_cache_t* cache, int32_t* total, int32_t* free_now);
 /* Frees the host handle (device memory stays the caller's). */
 int zz_cache_destroy(zz_cache_t* cache);
 /* Forgets the tokens of sequence `seq` (-1: all sequences) in every layer. */

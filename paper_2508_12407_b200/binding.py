@@ -62,6 +62,9 @@ SYMBOLS = {
     "zz_launch_count": (_i64, []),
     "zz_cache_query": (_i32, [_cfgp, ctypes.POINTER(_sz), ctypes.POINTER(_sz)]),
     "zz_cache_create": (_i32, [_cfgp, _vp, _sz, _vp, _sz, ctypes.POINTER(_vp)]),
+    "zz_cache_query_paged": (_i32, [_cfgp, _i32, ctypes.POINTER(_sz), ctypes.POINTER(_sz)]),
+    "zz_cache_create_paged": (_i32, [_cfgp, _i32, _vp, _sz, _vp, _sz, ctypes.POINTER(_vp)]),
+    "zz_cache_pages": (_i32, [_vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]),
     "zz_cache_destroy": (_i32, [_vp]),
     "zz_cache_reset": (_i32, [_vp, _i32, _vp]),
     "zz_cache_len": (_i32, [_vp, _i32, _i32, ctypes.POINTER(ctypes.c_int32)]),
@@ -174,7 +177,7 @@ class ZigzagCache:
                  recent: int, layer_is_retrieval: Sequence[int], capacity: Sequence[int],
                  max_new_tokens: int, softmax_scale: Optional[float] = None,
                  kvhead_is_retrieval: Optional[np.ndarray] = None, head_dim: int = 128,
-                 device: str = "cuda:0"):
+                 device: str = "cuda:0", pool_pages: int = 0):
         import torch
         lib = load()
         self._lib = lib
@@ -195,16 +198,26 @@ class ZigzagCache:
                        self._cap.ctypes.data)
         self._cfg = cfg
         a, w = ctypes.c_size_t(0), ctypes.c_size_t(0)
-        _check(lib.zz_cache_query(ctypes.byref(cfg), ctypes.byref(a), ctypes.byref(w)), "zz_cache_query")
+        self.pool_pages = int(pool_pages)
+        if self.pool_pages:
+            _check(lib.zz_cache_query_paged(ctypes.byref(cfg), self.pool_pages, ctypes.byref(a), ctypes.byref(w)),
+                   "zz_cache_query_paged")
+        else:
+            _check(lib.zz_cache_query(ctypes.byref(cfg), ctypes.byref(a), ctypes.byref(w)), "zz_cache_query")
         self.arena_bytes, self.workspace_bytes = int(a.value), int(w.value)
         self.device = torch.device(device)
         with torch.cuda.device(self.device):
             self._arena = torch.empty(self.arena_bytes, dtype=torch.uint8, device=self.device)
             self._work = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=self.device)
             h = ctypes.c_void_p(None)
-            _check(lib.zz_cache_create(ctypes.byref(cfg), self._arena.data_ptr(), self.arena_bytes,
-                                       self._work.data_ptr(), self.workspace_bytes, ctypes.byref(h)),
-                   "zz_cache_create")
+            if self.pool_pages:
+                _check(lib.zz_cache_create_paged(ctypes.byref(cfg), self.pool_pages, self._arena.data_ptr(),
+                                                 self.arena_bytes, self._work.data_ptr(), self.workspace_bytes,
+                                                 ctypes.byref(h)), "zz_cache_create_paged")
+            else:
+                _check(lib.zz_cache_create(ctypes.byref(cfg), self._arena.data_ptr(), self.arena_bytes,
+                                           self._work.data_ptr(), self.workspace_bytes, ctypes.byref(h)),
+                       "zz_cache_create")
         self._h = h
 
     # -- lifetime ---------------------------------------------------------------------------
@@ -229,6 +242,12 @@ class ZigzagCache:
         v = ctypes.c_int32(0)
         _check(self._lib.zz_cache_len(self._h, layer, seq, ctypes.byref(v)), "zz_cache_len")
         return int(v.value)
+
+    def pages(self):
+        """(pages in the pool, pages free now); (0, 0) for a cache with contiguous retrieval stores."""
+        t, f = ctypes.c_int32(0), ctypes.c_int32(0)
+        _check(self._lib.zz_cache_pages(self._h, ctypes.byref(t), ctypes.byref(f)), "zz_cache_pages")
+        return int(t.value), int(f.value)
 
     def tune(self, key: str, value: int) -> None:
         _check(self._lib.zz_tune(self._h, key.encode(), int(value)), "zz_tune")

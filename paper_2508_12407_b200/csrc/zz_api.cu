@@ -63,8 +63,9 @@ size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 struct Layout {
     // workspace sections (byte offsets)
     size_t off_status, off_len, off_pos, off_desc, off_heads, off_counters, off_part_ml, off_part_o,
-        off_qc, off_oc, off_dqc, off_doc, off_layer_ids, work_bytes;
+        off_qc, off_oc, off_dqc, off_doc, off_layer_ids, off_table, work_bytes;
     size_t arena_bytes, counters_per_layer, items_per_layer;
+    long long table_entries;   // page-table entries (0: contiguous retrieval stores)
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -136,6 +137,13 @@ struct zz_cache {
     int decode_multi_waves;
     bool last_nowait;   // the last launch did not wait for its predecessor: the next one must be an ordinary launch
     bool has_mixed;
+    // paged retrieval stores
+    bool paged;
+    int pool_pages;
+    std::vector<int> free_pages;      // stack of free page ids
+    std::vector<int> h_table;         // host mirror of the page table
+    std::vector<int> pages_of;        // [L*B] token blocks that already have pages
+    bool table_dirty;                 // page-table writes were launched: the next decode launch is an ordinary one
     alignas(64) CUtensorMap tmap_arena;
     bool have_tmap_arena;
 
@@ -145,6 +153,7 @@ struct zz_cache {
     int* d_pos(int l) const { return reinterpret_cast<int*>(work + lay.off_pos) + (size_t)l * B * ring; }
     SeqDesc* d_desc(int l) const { return reinterpret_cast<SeqDesc*>(work + lay.off_desc) + (size_t)l * B; }
     int* d_layer_ids() const { return reinterpret_cast<int*>(work + lay.off_layer_ids); }
+    int* d_table() const { return reinterpret_cast<int*>(work + lay.off_table); }
     int* d_heads(int l) const { return reinterpret_cast<int*>(work + lay.off_heads) + (size_t)l * Hkv; }
     unsigned int* d_counters(int l) const {
         return reinterpret_cast<unsigned int*>(work + lay.off_counters) + (size_t)l * lay.counters_per_layer;
@@ -188,11 +197,13 @@ uint8_t kind_of(const zz_config_t* c, int l, int h) {
 
 // Arena: for each layer, for each sequence: retrieval group K [nR][cap][128], V likewise, then
 // streaming group K [nS][S+W][128], V likewise.  Fills `desc` if given.
-void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* desc) {
+void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* desc, long long pool_pages = 0) {
     const int L = c->n_layers, B = c->batch, Hkv = c->n_kv_heads, Hq = c->n_q_heads;
     const int ring = c->sink + c->recent;
     const int G = Hq / Hkv;
     long long off = 0;  // elements
+    long long tbl = 0;  // page-table entries
+    const bool paged = pool_pages > 0;
     bool has_mixed = false;
     if (desc) desc->assign((size_t)L * B, SeqDesc());
     for (int l = 0; l < L; ++l) {
@@ -203,11 +214,17 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
         for (int b = 0; b < B; ++b) {
             SeqDesc d;
             d.cap = c->capacity[b];
-            d.pad = 0;
-            d.k_off[ZZ_KIND_RETRIEVAL] = off;
-            off += (long long)nR * d.cap * kD;
-            d.v_off[ZZ_KIND_RETRIEVAL] = off;
-            off += (long long)nR * d.cap * kD;
+            d.tbl = (int)tbl;
+            if (paged) {
+                // retrieval rows live in the pool (offsets filled in below): entries [token block][head]
+                tbl += (long long)((d.cap + zz::kPageTokens - 1) / zz::kPageTokens) * nR;
+                d.k_off[ZZ_KIND_RETRIEVAL] = d.v_off[ZZ_KIND_RETRIEVAL] = 0;
+            } else {
+                d.k_off[ZZ_KIND_RETRIEVAL] = off;
+                off += (long long)nR * d.cap * kD;
+                d.v_off[ZZ_KIND_RETRIEVAL] = off;
+                off += (long long)nR * d.cap * kD;
+            }
             d.k_off[ZZ_KIND_STREAMING] = off;
             off += (long long)nS * ring * kD;
             d.v_off[ZZ_KIND_STREAMING] = off;
@@ -215,6 +232,17 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
             if (desc) (*desc)[(size_t)l * B + b] = d;
         }
     }
+    if (paged) {
+        // the pool follows the rings; every descriptor points at it
+        const long long pool_off = off;
+        off += pool_pages * zz::kPageElems;
+        if (desc)
+            for (auto& d : *desc) {
+                d.k_off[ZZ_KIND_RETRIEVAL] = pool_off;
+                d.v_off[ZZ_KIND_RETRIEVAL] = pool_off + (long long)zz::kPageTokens * kD;
+            }
+    }
+    lay->table_entries = paged ? tbl : 0;
     // one spare tile of rows so that a 128-row tile read starting at the last valid row of the
     // last store stays inside the tensor map's extent (out-of-extent rows read as zero anyway)
     lay->arena_bytes = align_up((size_t)off * 2 + 128 * kD * 2);
@@ -225,6 +253,7 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
     lay->off_desc = w; w += align_up((size_t)L * B * sizeof(SeqDesc));
     lay->off_heads = w; w += align_up((size_t)L * Hkv * sizeof(int));
     lay->off_layer_ids = w; w += align_up((size_t)L * sizeof(int));
+    lay->off_table = w; w += align_up((size_t)lay->table_entries * sizeof(int));
     // per layer: arrival counters and the split partials of the layer's launches, indexed by work
     // item (at most kMaxSlots + B * Hkv items per launch), so that the launches of different
     // layers share no scratch and may overlap
@@ -292,8 +321,66 @@ void plan_splits(const zz_cache* c, const int* n, int Hg, int* warps, int* chunk
         if (s < 1) s = 1;
         chunk[b] = (n[b] + s - 1) / s;            // equal splits inside the sequence
         if (chunk[b] < 1) chunk[b] = 1;
+        if (c->paged) {
+            // splits start at multiples of 16 tokens, so that no 16-token block straddles a page
+            chunk[b] = (chunk[b] + 15) / 16 * 16;
+            s = (n[b] + chunk[b] - 1) / chunk[b];
+            if (s < 1) s = 1;
+        }
         split_start[b + 1] = split_start[b] + s;
     }
+}
+
+// Paged stores: make sure that layers [l0, l1) have pages for `add[b]` more tokens per sequence.
+// All or nothing: when the pool cannot cover the request nothing is taken and nothing is launched.
+// The new table entries reach the device through small kernels on the caller's stream (values
+// passed by value), so they are ordered before the launches that follow and no host buffer has to
+// stay untouched afterwards.
+int reserve_pages(zz_cache* c, int l0, int l1, const int32_t* add, cudaStream_t st) {
+    if (!c->paged) return ZZ_OK;
+    long long need = 0;
+    for (int l = l0; l < l1; ++l) {
+        if (c->nR[l] == 0) continue;
+        for (int b = 0; b < c->B; ++b) {
+            const long long nl = (long long)c->len[(size_t)l * c->B + b] + add[b];
+            const long long blocks = (nl + zz::kPageTokens - 1) / zz::kPageTokens - c->pages_of[(size_t)l * c->B + b];
+            if (blocks > 0) need += blocks * c->nR[l];
+        }
+    }
+    if (need == 0) return ZZ_OK;
+    if (need > (long long)c->free_pages.size()) return ZZ_ERR_CAPACITY;
+    zz::TableUpdate u;
+    u.n = 0;
+    auto flush = [&]() -> bool {
+        if (u.n == 0) return true;
+        const bool ok = zz::launch_table_update(c->d_table(), u, st) == cudaSuccess;
+        u.n = 0;
+        return ok;
+    };
+    for (int l = l0; l < l1; ++l) {
+        const int nR = c->nR[l];
+        if (nR == 0) continue;
+        for (int b = 0; b < c->B; ++b) {
+            const size_t lb = (size_t)l * c->B + b;
+            const long long nl = (long long)c->len[lb] + add[b];
+            const int want = (int)((nl + zz::kPageTokens - 1) / zz::kPageTokens);
+            for (int g = c->pages_of[lb]; g < want; ++g)
+                for (int h = 0; h < nR; ++h) {
+                    const int page = c->free_pages.back();
+                    c->free_pages.pop_back();
+                    const int idx = c->desc[lb].tbl + g * nR + h;
+                    c->h_table[idx] = page;
+                    u.idx[u.n] = idx;
+                    u.val[u.n] = page;
+                    if (++u.n == 480 && !flush()) return ZZ_ERR_CUDA;
+                }
+            if (want > c->pages_of[lb]) c->pages_of[lb] = want;
+        }
+    }
+    if (!flush()) return ZZ_ERR_CUDA;
+    c->table_dirty = true;
+    c->last_nowait = false;   // the table writes were ordinary launches
+    return ZZ_OK;
 }
 
 // k_new/v_new != nullptr: fused append of one token per sequence (host lengths not yet bumped)
@@ -333,6 +420,7 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
     p.B = c->B;
     p.max_splits = kMaxSplits;
     p.scale_log2 = c->scale * 1.4426950408889634f;
+    p.page_table = c->paged ? c->d_table() : nullptr;
     int n[ZZ_MAX_BATCH];
     for (int b = 0; b < c->B; ++b) {
         const int len = c->len[(size_t)layer * c->B + b] + (k_new ? 1 : 0);
@@ -347,6 +435,9 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
     // that did not wait for its own predecessor, only an ordinary launch (full stream order) or
     // another launch of the same independent chain may follow.
     if (c->last_nowait && overlap != 2) overlap = 0;
+    // page-table writes precede this launch as ordinary launches: read them in full stream order
+    if (c->table_dirty) overlap = 0;
+    c->table_dirty = false;
     c->last_nowait = (overlap == 2);
     if (d_layer_ids) {
         // one launch for n_multi layers with identical lengths: `layer` stands for all of them in the
@@ -411,6 +502,7 @@ int launch_prefill_group(zz_cache* c, int layer, int kind, const CUtensorMap* tq
     p.out = out;
     p.tok_stride = (long long)c->Hq * kD;
     p.head_list = c->d_heads(layer);
+    p.page_table = c->paged ? c->d_table() : nullptr;
     p.status = c->d_status();
     p.kind = kind;
     p.kv_head0 = (kind == ZZ_KIND_RETRIEVAL) ? 0 : nR;
@@ -466,19 +558,50 @@ const char* zz_status_str(int s) {
 
 int64_t zz_launch_count(void) { return zz::g_launches.load(std::memory_order_relaxed); }
 
-int zz_cache_query(const zz_config_t* cfg, size_t* arena_bytes, size_t* workspace_bytes) {
+static int query_impl(const zz_config_t* cfg, long long pool_pages, size_t* arena_bytes, size_t* workspace_bytes) {
     const int v = validate(cfg);
     if (v != ZZ_OK) return v;
     if (!arena_bytes || !workspace_bytes) return ZZ_ERR_INVALID_ARG;
     Layout lay;
-    compute_layout(cfg, &lay, nullptr);
+    compute_layout(cfg, &lay, nullptr, pool_pages);
+    if (lay.table_entries > 0x7fffffffLL) return ZZ_ERR_UNSUPPORTED;
     *arena_bytes = lay.arena_bytes;
     *workspace_bytes = lay.work_bytes;
     return ZZ_OK;
 }
 
+int zz_cache_query(const zz_config_t* cfg, size_t* arena_bytes, size_t* workspace_bytes) {
+    return query_impl(cfg, 0, arena_bytes, workspace_bytes);
+}
+
+int zz_cache_query_paged(const zz_config_t* cfg, int32_t pool_pages, size_t* arena_bytes, size_t* workspace_bytes) {
+    if (pool_pages < 1) return ZZ_ERR_INVALID_ARG;
+    return query_impl(cfg, pool_pages, arena_bytes, workspace_bytes);
+}
+
+static int create_impl(const zz_config_t* cfg, long long pool_pages, void* d_arena, size_t arena_bytes,
+                       void* d_workspace, size_t workspace_bytes, zz_cache_t** out);
+
 int zz_cache_create(const zz_config_t* cfg, void* d_arena, size_t arena_bytes, void* d_workspace,
                     size_t workspace_bytes, zz_cache_t** out) {
+    return create_impl(cfg, 0, d_arena, arena_bytes, d_workspace, workspace_bytes, out);
+}
+
+int zz_cache_create_paged(const zz_config_t* cfg, int32_t pool_pages, void* d_arena, size_t arena_bytes,
+                          void* d_workspace, size_t workspace_bytes, zz_cache_t** out) {
+    if (pool_pages < 1) return ZZ_ERR_INVALID_ARG;
+    return create_impl(cfg, pool_pages, d_arena, arena_bytes, d_workspace, workspace_bytes, out);
+}
+
+int zz_cache_pages(const zz_cache_t* c, int32_t* total, int32_t* free_now) {
+    if (!c || !total || !free_now) return ZZ_ERR_INVALID_ARG;
+    *total = c->paged ? c->pool_pages : 0;
+    *free_now = c->paged ? (int32_t)c->free_pages.size() : 0;
+    return ZZ_OK;
+}
+
+static int create_impl(const zz_config_t* cfg, long long pool_pages, void* d_arena, size_t arena_bytes,
+                       void* d_workspace, size_t workspace_bytes, zz_cache_t** out) {
     const int v = validate(cfg);
     if (v != ZZ_OK) return v;
     if (!d_arena || !d_workspace || !out) return ZZ_ERR_INVALID_ARG;
@@ -493,10 +616,23 @@ int zz_cache_create(const zz_config_t* cfg, void* d_arena, size_t arena_bytes, v
     c->decode_overlap = 3;
     c->last_nowait = false;
     c->decode_multi_waves = 8;
-    compute_layout(cfg, &c->lay, &c->desc);
+    compute_layout(cfg, &c->lay, &c->desc, pool_pages);
+    if (c->lay.table_entries > 0x7fffffffLL) {
+        delete c;
+        return ZZ_ERR_UNSUPPORTED;
+    }
     if (arena_bytes < c->lay.arena_bytes || workspace_bytes < c->lay.work_bytes) {
         delete c;
         return ZZ_ERR_WORKSPACE;
+    }
+    c->paged = pool_pages > 0;
+    c->pool_pages = (int)pool_pages;
+    c->table_dirty = false;
+    if (c->paged) {
+        c->h_table.assign((size_t)c->lay.table_entries, 0);
+        c->pages_of.assign((size_t)c->L * c->B, 0);
+        c->free_pages.resize((size_t)pool_pages);
+        for (long long i = 0; i < pool_pages; ++i) c->free_pages[(size_t)i] = (int)(pool_pages - 1 - i);  // page 0 on top
     }
     c->arena = static_cast<unsigned char*>(d_arena);
     c->work = static_cast<unsigned char*>(d_workspace);
@@ -575,7 +711,17 @@ int zz_cache_reset(zz_cache_t* c, int seq, void* stream) {
         return ZZ_ERR_CUDA;
     for (int l = 0; l < c->L; ++l)
         for (int b = 0; b < c->B; ++b)
-            if (seq < 0 || seq == b) c->len[(size_t)l * c->B + b] = 0;
+            if (seq < 0 || seq == b) {
+                const size_t lb = (size_t)l * c->B + b;
+                c->len[lb] = 0;
+                if (c->paged) {
+                    // the sequence's pages go back to the pool (work already in the stream that reads
+                    // them is ordered before whatever writes them next on the same stream)
+                    const int n = c->pages_of[lb] * c->nR[l];
+                    for (int i = 0; i < n; ++i) c->free_pages.push_back(c->h_table[c->desc[lb].tbl + i]);
+                    c->pages_of[lb] = 0;
+                }
+            }
     return ZZ_OK;
 }
 
@@ -624,6 +770,10 @@ int zz_kv_append(zz_cache_t* c, int layer, const void* d_k, const void* d_v, con
         total += h_n_new[b];
     }
     if (total == 0) return ZZ_OK;
+    {
+        const int rp = reserve_pages(c, layer, layer + 1, h_n_new, static_cast<cudaStream_t>(stream));
+        if (rp != ZZ_OK) return rp;
+    }
     zz::AppendParams p;
     memset(&p, 0, sizeof p);
     p.arena = c->d_arena();
@@ -634,6 +784,7 @@ int zz_kv_append(zz_cache_t* c, int layer, const void* d_k, const void* d_v, con
     p.k_new = static_cast<const __nv_bfloat16*>(d_k);
     p.v_new = static_cast<const __nv_bfloat16*>(d_v);
     p.head_list = c->d_heads(layer);
+    p.page_table = c->paged ? c->d_table() : nullptr;
     p.nR = nR; p.Hkv = c->Hkv; p.ring = c->ring; p.S = c->S; p.W = c->W; p.B = c->B;
     int off = 0;
     for (int b = 0; b < c->B; ++b) {
@@ -700,6 +851,12 @@ static int decode_step_impl(zz_cache_t* c, int layer, const void* d_q, const voi
     // the append is fused into the attention kernel: the new row is read from d_k/d_v, stored in
     // its slot and attended to by the same launch
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    {
+        int32_t ones[ZZ_MAX_BATCH];
+        for (int b = 0; b < c->B; ++b) ones[b] = 1;
+        const int rp = reserve_pages(c, layer, layer + 1, ones, st);
+        if (rp != ZZ_OK) return rp;
+    }
     const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(d_q);
     const __nv_bfloat16* k = static_cast<const __nv_bfloat16*>(d_k);
     const __nv_bfloat16* v = static_cast<const __nv_bfloat16*>(d_v);
@@ -730,6 +887,12 @@ int zz_decode_step_all(zz_cache_t* c, const void* d_q, const void* d_k, const vo
     for (int l = 0; l < c->L; ++l)
         for (int b = 0; b < c->B; ++b)
             if (c->nR[l] > 0 && c->len[(size_t)l * c->B + b] + 1 > c->cap[b]) return ZZ_ERR_CAPACITY;
+    {
+        int32_t ones[ZZ_MAX_BATCH];
+        for (int b = 0; b < c->B; ++b) ones[b] = 1;
+        const int rp = reserve_pages(c, 0, c->L, ones, static_cast<cudaStream_t>(stream));
+        if (rp != ZZ_OK) return rp;
+    }
     // Equal lengths in every layer: one launch per kind of work instead of one (or four) per layer
     // (blockIdx.y = layer).  The layers are independent (own stores, lengths, scratch and output
     // slice; q/k/v of all layers are inputs of the call), so a launch over many layers only removes
@@ -950,7 +1113,22 @@ int zz_cache_export(zz_cache_t* c, int layer, int seq, int kind, void* h_k, void
     const SeqDesc& d = c->desc[(size_t)layer * c->B + seq];
     const size_t bytes = (size_t)nh * ns * kD * 2;
     cudaError_t e = cudaSuccess;
-    if (bytes) {
+    if (bytes && c->paged && kind == ZZ_KIND_RETRIEVAL) {
+        // page by page into the contiguous [head][slot][128] host layout; slots without a page are left alone
+        const size_t lb = (size_t)layer * c->B + seq;
+        for (int g = 0; g < c->pages_of[lb] && e == cudaSuccess; ++g)
+            for (int h = 0; h < nh && e == cudaSuccess; ++h) {
+                const long long page = c->h_table[d.tbl + g * nh + h];
+                const int rows = (ns - g * zz::kPageTokens < zz::kPageTokens) ? ns - g * zz::kPageTokens : zz::kPageTokens;
+                const size_t ho = ((size_t)h * ns + (size_t)g * zz::kPageTokens) * kD * 2;
+                e = cudaMemcpyAsync(static_cast<char*>(h_k) + ho, c->d_arena() + d.k_off[kind] + page * zz::kPageElems,
+                                    (size_t)rows * kD * 2, cudaMemcpyDeviceToHost, st);
+                if (e == cudaSuccess)
+                    e = cudaMemcpyAsync(static_cast<char*>(h_v) + ho,
+                                        c->d_arena() + d.v_off[kind] + page * zz::kPageElems, (size_t)rows * kD * 2,
+                                        cudaMemcpyDeviceToHost, st);
+            }
+    } else if (bytes) {
         e = cudaMemcpyAsync(h_k, c->d_arena() + d.k_off[kind], bytes, cudaMemcpyDeviceToHost, st);
         if (e == cudaSuccess) e = cudaMemcpyAsync(h_v, c->d_arena() + d.v_off[kind], bytes, cudaMemcpyDeviceToHost, st);
     }
@@ -978,7 +1156,26 @@ int zz_cache_import(zz_cache_t* c, int layer, int seq, int kind, const void* h_k
     const SeqDesc& d = c->desc[(size_t)layer * c->B + seq];
     const size_t bytes = (size_t)nh * ns * kD * 2;
     cudaError_t e = cudaSuccess;
-    if (bytes) {
+    if (bytes && c->paged && kind == ZZ_KIND_RETRIEVAL) {
+        const size_t lb = (size_t)layer * c->B + seq;
+        int32_t add[ZZ_MAX_BATCH] = {0};
+        add[seq] = len > c->len[lb] ? len - c->len[lb] : 0;
+        const int rp = reserve_pages(c, layer, layer + 1, add, st);
+        if (rp != ZZ_OK) return rp;
+        const int blocks = (len + zz::kPageTokens - 1) / zz::kPageTokens;
+        for (int g = 0; g < blocks && e == cudaSuccess; ++g)
+            for (int h = 0; h < nh && e == cudaSuccess; ++h) {
+                const long long page = c->h_table[d.tbl + g * nh + h];
+                const int rows = (ns - g * zz::kPageTokens < zz::kPageTokens) ? ns - g * zz::kPageTokens : zz::kPageTokens;
+                const size_t ho = ((size_t)h * ns + (size_t)g * zz::kPageTokens) * kD * 2;
+                e = cudaMemcpyAsync(c->d_arena() + d.k_off[kind] + page * zz::kPageElems,
+                                    static_cast<const char*>(h_k) + ho, (size_t)rows * kD * 2, cudaMemcpyHostToDevice, st);
+                if (e == cudaSuccess)
+                    e = cudaMemcpyAsync(c->d_arena() + d.v_off[kind] + page * zz::kPageElems,
+                                        static_cast<const char*>(h_v) + ho, (size_t)rows * kD * 2,
+                                        cudaMemcpyHostToDevice, st);
+            }
+    } else if (bytes) {
         e = cudaMemcpyAsync(c->d_arena() + d.k_off[kind], h_k, bytes, cudaMemcpyHostToDevice, st);
         if (e == cudaSuccess) e = cudaMemcpyAsync(c->d_arena() + d.v_off[kind], h_v, bytes, cudaMemcpyHostToDevice, st);
     }

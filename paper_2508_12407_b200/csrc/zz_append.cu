@@ -52,7 +52,12 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendParams p) {
         const int src_head = p.head_list[(kind == ZZ_KIND_RETRIEVAL) ? hi : p.nR + hi];
         const long long slots_per_head = (kind == ZZ_KIND_RETRIEVAL) ? sd.cap : p.ring;
         const long long src = ((long long)(p.tok_off[b] + i) * p.Hkv + src_head) * kD + piece * 8;
-        const long long dst = ((long long)hi * slots_per_head + slot) * kD + piece * 8;
+        long long dst = ((long long)hi * slots_per_head + slot) * kD + piece * 8;
+        if (kind == ZZ_KIND_RETRIEVAL && p.page_table) {
+            // paged store: the slot's page comes from the table (K rows, then V rows, per page)
+            const int page = p.page_table[sd.tbl + (int)(slot >> 7) * p.nR + hi];
+            dst = (long long)page * kPageElems + (slot & (kPageTokens - 1)) * kD + piece * 8;
+        }
         const uint4 kk = *reinterpret_cast<const uint4*>(p.k_new + src);
         const uint4 vv = *reinterpret_cast<const uint4*>(p.v_new + src);
         *reinterpret_cast<uint4*>(p.arena + sd.k_off[kind] + dst) = kk;
@@ -130,6 +135,18 @@ __global__ void __launch_bounds__(256) regroup_kernel(const GatherParams p) {
         else
             *reinterpret_cast<uint4*>(p.dst + model) = *reinterpret_cast<const uint4*>(p.src + compact);
     }
+}
+
+// Page-table entries of newly allocated pages (at most 480 per launch, passed by value).
+__global__ void __launch_bounds__(512) table_update_kernel(int* table, const TableUpdate u) {
+    const int i = threadIdx.x;
+    if (i < u.n) table[u.idx[i]] = u.val[i];
+}
+
+cudaError_t launch_table_update(int* table, const TableUpdate& u, cudaStream_t s) {
+    table_update_kernel<<<1, 512, 0, s>>>(table, u);
+    count_launch();
+    return cudaGetLastError();
 }
 
 cudaError_t launch_regroup(const GatherParams& p, cudaStream_t s, int programmatic) {

@@ -16,11 +16,26 @@ constexpr int kRowBytes = kD * 2;  // one K or V row of one head
 // Where the stores of one (layer, sequence) live in the arena, in bf16 elements from the
 // arena base.  Index [ZZ_KIND_STREAMING] is the ring group, [ZZ_KIND_RETRIEVAL] the
 // append-only group; each group is laid out [head_in_group][slot][128].
+//
+// Paged retrieval stores (a cache built with a page pool): a page holds 128 tokens of one KV
+// head, its K rows [128][128] followed by its V rows.  k_off[ZZ_KIND_RETRIEVAL] is then the
+// pool's first K row, v_off[...] the first V row (128 rows further), and the page of token t of
+// head h is page_table[tbl + (t / 128) * n_retrieval_heads + h].
 struct SeqDesc {
     long long k_off[2];
     long long v_off[2];
     int cap;   // slots per head of the retrieval group (capacity of this sequence)
-    int pad;
+    int tbl;   // paged stores: first page-table entry of this (layer, sequence)
+};
+
+constexpr int kPageTokens = 128;
+constexpr long long kPageElems = 2LL * kPageTokens * kD;   // K block, then V block
+
+// Page-table writes of one launch (passed by value: no host buffer has to outlive the call).
+struct TableUpdate {
+    int n;
+    int idx[480];
+    int val[480];
 };
 
 struct AppendParams {
@@ -32,6 +47,7 @@ struct AppendParams {
     const __nv_bfloat16* k_new;  // [sum n_new][Hkv][128]
     const __nv_bfloat16* v_new;
     const int* head_list;    // [Hkv] source KV heads: first nR retrieval heads, then streaming
+    const int* page_table;   // nullptr: contiguous retrieval stores
     int nR, Hkv, ring, S, W, B;
     int n_new[ZZ_MAX_BATCH];
     int tok_off[ZZ_MAX_BATCH];
@@ -74,6 +90,7 @@ struct DecodeParams {
     // store addresses come from desc_table[layer * B + b].  layer_ids == nullptr: one layer.
     const int* layer_ids;
     const SeqDesc* desc_table;
+    const int* page_table;   // nullptr: contiguous retrieval stores
     long long st_len, st_pos, st_q, st_kv, st_cnt, st_part;
 };
 
@@ -97,7 +114,7 @@ struct PrefillParams {
     const int* pos;          // [B][ring] ring positions of this layer
     __nv_bfloat16* out;      // row of packed token i, head h at out + i*tok_stride + (q_head0+h)*128
     long long tok_stride;    // n_q_heads * 128
-    long long arena_row0;    // unused by the kernel (rows are derived from desc offsets)
+    const int* page_table;   // nullptr: contiguous retrieval stores
     const int* head_list;    // [Hkv] group-ordered source KV heads (for the chunk K/V)
     int* status;
     int kind;                // group served by this launch
@@ -118,6 +135,7 @@ cudaError_t launch_append(const AppendParams& p, int grid_x, cudaStream_t s);
 cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStream_t s, int overlap = 0, int n_layers = 1);
 cudaError_t launch_regroup(const GatherParams& p, cudaStream_t s, int programmatic);
 cudaError_t launch_reset(int* len, int* pos, int L, int B, int ring, int seq, cudaStream_t s);
+cudaError_t launch_table_update(int* table, const TableUpdate& u, cudaStream_t s);
 cudaError_t decode_setup();
 cudaError_t prefill_setup();
 // tensor maps: q [tokens][heads][128] (3-D), chunk k and v [tokens][kv heads][128] (3-D), and the

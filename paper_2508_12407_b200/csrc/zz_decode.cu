@@ -100,7 +100,8 @@ __device__ __forceinline__ void load_block(uint32_t stage_k, uint32_t stage_v, c
 }
 
 // HI = group size above 8 (rows 8..15 of the tile carry query heads too).
-template <bool HI, int kWarps>
+// kPaged: the retrieval store is paged (compiled apart, so that the contiguous kernel carries none of it).
+template <bool HI, int kWarps, bool kPaged>
 __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const DecodeParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     __shared__ int s_is_last;
@@ -145,8 +146,11 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     const int len = len_old + (fused ? 1 : 0);
     const int n = (p.kind == ZZ_KIND_RETRIEVAL) ? len : min(len, p.ring);
     const long long slots_per_head = (p.kind == ZZ_KIND_RETRIEVAL) ? sd.cap : p.ring;
-    __nv_bfloat16* kbase = p.arena + sd.k_off[p.kind] + (long long)hg * slots_per_head * kD;
-    __nv_bfloat16* vbase = p.arena + sd.v_off[p.kind] + (long long)hg * slots_per_head * kD;
+    // paged retrieval store: the bases are the pool's; each 16-token block adds its page's offset
+    constexpr bool paged = kPaged;
+    __nv_bfloat16* kbase = p.arena + sd.k_off[p.kind] + (paged ? 0ll : (long long)hg * slots_per_head * kD);
+    __nv_bfloat16* vbase = p.arena + sd.v_off[p.kind] + (paged ? 0ll : (long long)hg * slots_per_head * kD);
+    const int* const tbl = paged ? p.page_table + sd.tbl + hg : nullptr;   // entry of page g: tbl[g * Hg]
     int new_slot = -1;
     const __nv_bfloat16* knew = nullptr;
     const __nv_bfloat16* vnew = nullptr;
@@ -167,7 +171,10 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     if (fused && new_slot >= s0 && new_slot < s1 && warp == kWarps - 1) {
         const int c = lane & 15;
         const __nv_bfloat16* src = (lane < 16 ? knew : vnew) + c * 8;
-        __nv_bfloat16* dst = (lane < 16 ? kbase : vbase) + (long long)new_slot * kD + c * 8;
+        long long slot_off = (long long)new_slot * kD;
+        if (paged)
+            slot_off = (long long)tbl[(new_slot >> 7) * p.Hg] * kPageElems + (new_slot & (kPageTokens - 1)) * kD;
+        __nv_bfloat16* dst = (lane < 16 ? kbase : vbase) + slot_off + c * 8;
         *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
         if (p.kind == ZZ_KIND_STREAMING && hg == 0 && lane == 0) pos_p[(long long)b * p.ring + new_slot] = len_old;
     }
@@ -200,12 +207,31 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
 
     const uint32_t wbase = smem_u32(smem) + warp * kWarpSmem;
 
+    // Paged store: lane i holds the page of token block pg0 + i (32 pages = 4096 tokens); a block's
+    // page is a shuffle away, the window is reloaded when the warp walks past it.  Blocks start at
+    // multiples of 16 tokens (the split plan of a paged cache guarantees it), so a block never
+    // straddles a page.  The offset returned maps token t of the block to its row: base + off + t*128.
+    const int n_pages = paged ? (sd.cap + kPageTokens - 1) / kPageTokens : 0;
+    int pg0 = s0 >> 7;
+    int win = (paged && pg0 + lane < n_pages) ? tbl[(pg0 + lane) * p.Hg] : 0;
+    auto page_off = [&](int tok0) -> long long {
+        if constexpr (!paged) return 0ll;
+        const int pg = tok0 >> 7;
+        if (pg - pg0 >= 32) {
+            pg0 = pg;
+            win = (pg0 + lane < n_pages) ? tbl[(pg0 + lane) * p.Hg] : 0;
+        }
+        const int page = __shfl_sync(0xffffffffu, win, pg - pg0);
+        return (long long)page * kPageElems - (long long)pg * kPageTokens * kD;
+    };
+
     // prologue: fill kStages-1 stages
 #pragma unroll
     for (int s = 0; s < kStages - 1; ++s) {
         if (s < my_blocks) {
             const int tok0 = s0 + (warp + s * kWarps) * kBlk;
-            load_block(wbase + s * 2 * kStageBytes, wbase + s * 2 * kStageBytes + kStageBytes, kbase, vbase,
+            const long long po = page_off(tok0);
+            load_block(wbase + s * 2 * kStageBytes, wbase + s * 2 * kStageBytes + kStageBytes, kbase + po, vbase + po,
                        tok0, s1, lane, new_slot, knew, vnew);
         }
         cp_async_commit();
@@ -217,8 +243,9 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
             if (nx < my_blocks) {
                 const int st = nx % kStages;
                 const int tok0 = s0 + (warp + nx * kWarps) * kBlk;
-                load_block(wbase + st * 2 * kStageBytes, wbase + st * 2 * kStageBytes + kStageBytes, kbase,
-                           vbase, tok0, s1, lane, new_slot, knew, vnew);
+                const long long po = page_off(tok0);
+                load_block(wbase + st * 2 * kStageBytes, wbase + st * 2 * kStageBytes + kStageBytes, kbase + po,
+                           vbase + po, tok0, s1, lane, new_slot, knew, vnew);
             }
             cp_async_commit();
         }
@@ -446,19 +473,21 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
 
 }  // namespace
 
+template <bool HI, int kWarps, bool kPaged>
+static cudaError_t setup_one() {
+    return cudaFuncSetAttribute(decode_kernel<HI, kWarps, kPaged>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                kWarps * kWarpSmem);
+}
+
 cudaError_t decode_setup() {
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel<false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         4 * kWarpSmem);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(decode_kernel<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * kWarpSmem);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(decode_kernel<false, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * kWarpSmem);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(decode_kernel<true, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * kWarpSmem);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(decode_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kWarpSmem);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(decode_kernel<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kWarpSmem);
+    cudaError_t e = setup_one<false, 4, false>();
+    if (e == cudaSuccess) e = setup_one<true, 4, false>();
+    if (e == cudaSuccess) e = setup_one<false, 8, false>();
+    if (e == cudaSuccess) e = setup_one<true, 8, false>();
+    if (e == cudaSuccess) e = setup_one<false, 4, true>();
+    if (e == cudaSuccess) e = setup_one<true, 4, true>();
+    if (e == cudaSuccess) e = setup_one<false, 8, true>();
+    if (e == cudaSuccess) e = setup_one<true, 8, true>();
     return e;
 }
 
@@ -483,17 +512,19 @@ cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStr
     cfg.numAttrs = overlap ? 1 : 0;
     DecodeParams pp = p;
     pp.gdc_wait = (overlap == 2) ? 0 : (overlap == 3) ? 2 : 1;
+    const bool paged = p.page_table != nullptr && p.kind == ZZ_KIND_RETRIEVAL;
+    const bool hi = p.G > 8;
     cudaError_t e;
+    if (warps != 4 && warps != 8) return cudaErrorInvalidValue;
+#define ZZ_LAUNCH(HI_, W_, PG_) e = cudaLaunchKernelEx(&cfg, decode_kernel<HI_, W_, PG_>, pp)
     if (warps == 8) {
-        if (p.G > 8) e = cudaLaunchKernelEx(&cfg, decode_kernel<true, 8>, pp);
-        else e = cudaLaunchKernelEx(&cfg, decode_kernel<false, 8>, pp);
-    } else if (warps == 2) {
-        if (p.G > 8) e = cudaLaunchKernelEx(&cfg, decode_kernel<true, 2>, pp);
-        else e = cudaLaunchKernelEx(&cfg, decode_kernel<false, 2>, pp);
+        if (paged) { if (hi) ZZ_LAUNCH(true, 8, true); else ZZ_LAUNCH(false, 8, true); }
+        else { if (hi) ZZ_LAUNCH(true, 8, false); else ZZ_LAUNCH(false, 8, false); }
     } else {
-        if (p.G > 8) e = cudaLaunchKernelEx(&cfg, decode_kernel<true, 4>, pp);
-        else e = cudaLaunchKernelEx(&cfg, decode_kernel<false, 4>, pp);
+        if (paged) { if (hi) ZZ_LAUNCH(true, 4, true); else ZZ_LAUNCH(false, 4, true); }
+        else { if (hi) ZZ_LAUNCH(true, 4, false); else ZZ_LAUNCH(false, 4, false); }
     }
+#undef ZZ_LAUNCH
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -411,8 +411,11 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                 const Item it = get_item(p, idx);
                 const SeqDesc sd = p.desc[it.b];
                 const long long slots_per_head = (p.kind == ZZ_KIND_RETRIEVAL) ? sd.cap : p.ring;
-                const int k_row0 = (int)(sd.k_off[p.kind] / kD + (long long)it.hg * slots_per_head);
-                const int v_row0 = (int)(sd.v_off[p.kind] / kD + (long long)it.hg * slots_per_head);
+                // paged retrieval store: a store tile is one page (tiles and pages are both 128 tokens)
+                const bool paged = p.page_table != nullptr && p.kind == ZZ_KIND_RETRIEVAL;
+                const int* const tbl = paged ? p.page_table + sd.tbl + it.hg : nullptr;
+                const int k_row0 = (int)(sd.k_off[p.kind] / kD + (paged ? 0ll : (long long)it.hg * slots_per_head));
+                const int v_row0 = (int)(sd.v_off[p.kind] / kD + (paged ? 0ll : (long long)it.hg * slots_per_head));
                 const int src_head = p.head_list[p.kv_head0 + it.hg];
                 const int tok0 = p.tok_off[it.b];
                 const int qh = p.q_head0 + it.hg * p.G + it.g0;
@@ -443,7 +446,8 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                             tma_load_3d(dst, m, 0, src_head, tok0 + start, &sh.kv_full[slot]);
                             tma_load_3d(dst + kSubBytes, m, 64, src_head, tok0 + start, &sh.kv_full[slot]);
                         } else {
-                            const int row = (is_k ? k_row0 : v_row0) + start;
+                            const int row = (is_k ? k_row0 : v_row0) +
+                                            (paged ? tbl[(start >> 7) * p.Hg] * (int)(kPageElems / kD) : start);
                             tma_load_2d(dst, &tmap_arena, 0, row, &sh.kv_full[slot]);
                             tma_load_2d(dst + kSubBytes, &tmap_arena, 64, row, &sh.kv_full[slot]);
                         }

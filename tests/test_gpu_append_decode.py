@@ -15,8 +15,9 @@ def _built():
     binding.load()
 
 
-def make(L, B, Hq, Hkv, S, W, kinds, cap, kvk=None, max_new=4096):
-    return binding.ZigzagCache(L, B, Hq, Hkv, S, W, kinds, cap, max_new, kvhead_is_retrieval=kvk)
+def make(L, B, Hq, Hkv, S, W, kinds, cap, kvk=None, max_new=4096, pool_pages=0):
+    return binding.ZigzagCache(L, B, Hq, Hkv, S, W, kinds, cap, max_new, kvhead_is_retrieval=kvk,
+                               pool_pages=pool_pages)
 
 
 def layer_kv_kinds(kinds, Hkv, kvk, l):
@@ -26,11 +27,11 @@ def layer_kv_kinds(kinds, Hkv, kvk, l):
 
 
 def run_append_decode(L, B, Hq, Hkv, S, W, kinds, lens, n_decode, seed, kvk=None, chunk_cap=300,
-                      check_every=1):
+                      check_every=1, pool_pages=0):
     D = 128
     scale = 1.0 / np.sqrt(D)
     cap = [int(n) + n_decode for n in lens]
-    cache = make(L, B, Hq, Hkv, S, W, kinds, cap, kvk)
+    cache = make(L, B, Hq, Hkv, S, W, kinds, cap, kvk, pool_pages=pool_pages)
     w = inputs.Workload("t", L, B, Hq, Hkv, D, S, W, int(sum(kinds)), 0, 0, n_decode, seed=seed)
     orc = [[OracleSeq(Hkv, D, S, W, cap[b], layer_kv_kinds(kinds, Hkv, kvk, l)) for b in range(B)]
            for l in range(L)]

@@ -29,14 +29,17 @@ def _rows(P, c, S, W, n_extra, rng):
 
 
 def run_full(w: inputs.Workload, kinds, lens, chunk, n_decode, kvk=None, prefilled=False, rows_per_call=6,
-             decode_seqs=None, same_prompt_all_layers=False):
+             decode_seqs=None, same_prompt_all_layers=False, paged=False):
     L, B, Hq, Hkv, S, W = len(kinds), len(lens), w.n_q_heads, w.n_kv_heads, w.sink, w.recent
     import torch
     scale = w.scale
     rng = np.random.default_rng(w.seed)
     cap = [int(n) + n_decode + 8 for n in lens]
     max_new = B * chunk if chunk else B
-    cache = binding.ZigzagCache(L, B, Hq, Hkv, S, W, kinds, cap, max_new, kvhead_is_retrieval=kvk)
+    kk = np.asarray(kvk).reshape(L, Hkv) if kvk is not None else np.repeat(np.asarray(kinds)[:, None], Hkv, axis=1)
+    # paged: a pool with exactly the pages the run needs (one per retrieval head per 128 tokens)
+    pool = int(kk.sum()) * sum((int(n) + n_decode + 127) // 128 for n in lens) if paged else 0
+    cache = binding.ZigzagCache(L, B, Hq, Hkv, S, W, kinds, cap, max_new, kvhead_is_retrieval=kvk, pool_pages=pool)
     kv_kinds = [list(np.asarray(kvk).reshape(L, Hkv)[l]) if kvk is not None else [int(kinds[l])] * Hkv
                 for l in range(L)]
     hist_k = [[np.zeros((cap[b], Hkv, D), np.uint16) for b in range(B)] for l in range(L)]
@@ -128,6 +131,8 @@ def run_full(w: inputs.Workload, kinds, lens, chunk, n_decode, kvk=None, prefill
                 assert np.array_equal(gk[:, sl], np.ascontiguousarray(hist_k[l][b][sl][:, r_heads]).transpose(1, 0, 2))
                 assert np.array_equal(gv[:, :2000], np.ascontiguousarray(hist_v[l][b][:2000][:, r_heads]).transpose(1, 0, 2))
     assert cache.last_status() == 0
+    if paged:
+        assert cache.pages()[1] == 0          # every page of the exactly sized pool is in use
     cache.close()
 
 
@@ -152,3 +157,15 @@ def test_cfg5_64k_batch4_exclusive_and_mixed():
     kvk = np.stack([np.ones(8, np.uint8), np.zeros(8, np.uint8), inputs.mixed_kvhead_kinds(w)[0]])
     run_full(w, [1, 0, 0], [w.prefill_len] * w.batch, w.prefill_chunk, 2, kvk=kvk, rows_per_call=2,
              decode_seqs=[0, 3], same_prompt_all_layers=True)
+
+
+def test_cfg3_128k_paged_stores():
+    # the same 8K-chunked 128K prefill and decode with the retrieval store in 128-token pages
+    w = inputs.WORKLOADS["cfg3"]
+    run_full(w, [1, 0], [w.prefill_len], w.prefill_chunk, 3, rows_per_call=1, paged=True)
+
+
+def test_cfg4_ragged_batch16_paged_stores():
+    w = inputs.WORKLOADS["cfg4"]
+    lens = [int(x) for x in inputs.ragged_lengths(w)]
+    run_full(w, [1, 0], lens, 0, 3, prefilled=True, decode_seqs=[0, 5, 11, 15], paged=True)

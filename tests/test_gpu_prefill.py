@@ -15,7 +15,8 @@ def _built():
     binding.load()
 
 
-def run_prefill(L, B, Hq, Hkv, S, W, kinds, chunk_plans, seed, kvk=None, n_decode=0, sample_rows=None):
+def run_prefill(L, B, Hq, Hkv, S, W, kinds, chunk_plans, seed, kvk=None, n_decode=0, sample_rows=None,
+                pool_pages=0):
     """chunk_plans[b] = list of chunk sizes of sequence b (a 0 skips the sequence in that call)."""
     D = 128
     scale = 1.0 / np.sqrt(D)
@@ -23,7 +24,8 @@ def run_prefill(L, B, Hq, Hkv, S, W, kinds, chunk_plans, seed, kvk=None, n_decod
     cap = [t + n_decode + 1 for t in total]
     max_new = max(sum(pl[r] if r < len(pl) else 0 for pl in chunk_plans)
                   for r in range(max(len(pl) for pl in chunk_plans)))
-    cache = binding.ZigzagCache(L, B, Hq, Hkv, S, W, kinds, cap, max(max_new, B), kvhead_is_retrieval=kvk)
+    cache = binding.ZigzagCache(L, B, Hq, Hkv, S, W, kinds, cap, max(max_new, B), kvhead_is_retrieval=kvk,
+                                pool_pages=pool_pages)
     w = inputs.Workload("t", L, B, Hq, Hkv, D, S, W, int(sum(kinds)), 0, 0, n_decode, seed=seed)
 
     def kv_kinds(l):
