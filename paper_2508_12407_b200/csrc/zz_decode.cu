@@ -38,6 +38,9 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int sr
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes)
                  : "memory");
 }
+__device__ __forceinline__ void cp_async16_full(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
@@ -85,6 +88,23 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ void load_block(uint32_t stage_k, uint32_t stage_v, const __nv_bfloat16* kbase,
                                            const __nv_bfloat16* vbase, int tok0, int tok_end, int lane,
                                            int new_slot, const __nv_bfloat16* knew, const __nv_bfloat16* vnew) {
+    if (tok0 + kBlk <= tok_end && (new_slot < tok0 || new_slot >= tok0 + kBlk)) {
+        // Whole block from the store (all but the edge blocks of a range): one pointer per lane, every
+        // further address a constant away.  Row r = 2*it + r0 swizzles with (r & 7) = 2*(it & 3) + r0,
+        // which touches bits the two terms do not share, so it folds into one XOR per iteration.
+        const int r0 = lane >> 4, c = lane & 15;
+        const long long off0 = (long long)(tok0 + r0) * kD + c * 8;
+        const __nv_bfloat16* kp = kbase + off0;
+        const __nv_bfloat16* vp = vbase + off0;
+        const uint32_t so0 = r0 * kRowBytes + ((c ^ r0) << 4);
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const uint32_t so = (so0 ^ ((it & 3) << 5)) + it * 2 * kRowBytes;
+            cp_async16_full(stage_k + so, kp + it * 2 * kD);
+            cp_async16_full(stage_v + so, vp + it * 2 * kD);
+        }
+        return;
+    }
 #pragma unroll
     for (int it = 0; it < 8; ++it) {
         const int idx = it * 32 + lane;

@@ -27,6 +27,7 @@ def main():
     ap.add_argument("--layers", type=int, default=2)
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--recent", type=int, default=256)
+    ap.add_argument("--paged", action="store_true", help="retrieval stores in 128-token pages")
     args = ap.parse_args()
     build.build()
     binding.load()
@@ -46,8 +47,10 @@ def main():
     kvk = None
     if args.case == "mixed":
         kvk = np.tile(np.array([1, 0, 1, 0, 0, 1, 1, 0], dtype=np.uint8), (L, 1))
+    heads_R = int(kvk.sum()) if kvk is not None else int(sum(kinds)) * Hkv
+    pool = heads_R * B * ((N + 64 + 127) // 128) if args.paged else 0
     cache = binding.ZigzagCache(L, B, Hq, Hkv, S, W, kinds, [N + 64] * B, max(B * N, B),
-                                kvhead_is_retrieval=kvk)
+                                kvhead_is_retrieval=kvk, pool_pages=pool)
     if args.case in ("prefill_r", "prefill_s"):
         q, k, v = randn(B * N, Hq, D), randn(B * N, Hkv, D), randn(B * N, Hkv, D)
         out = torch.empty_like(q)
