@@ -300,30 +300,41 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
 #pragma unroll
             for (int nt = 0; nt < 2; ++nt) {
 #pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int col = nt * 8 + tig * 2 + e;
-                    const float x = sc[nt][hf * 2 + e] * p.scale_log2;
-                    t[nt * 2 + e] = (col < valid) ? x : -INFINITY;
+                for (int e = 0; e < 2; ++e) t[nt * 2 + e] = sc[nt][hf * 2 + e];
+            }
+            if (valid < kBlk) {        // the last block of a range (warp-uniform)
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+                    for (int e = 0; e < 2; ++e)
+                        if (nt * 8 + tig * 2 + e >= valid) t[nt * 2 + e] = -INFINITY;
                 }
             }
+            // the scale is positive, so the maximum is taken on the raw scores
             float mx = fmaxf(fmaxf(t[0], t[1]), fmaxf(t[2], t[3]));
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-            const float m_new = fmaxf(m_run[hf], mx);      // finite: column 0 is always valid
-            const float alpha = fast_exp2(m_run[hf] - m_new);  // 0 on the first block
+            const float m_new = fmaxf(m_run[hf], mx * p.scale_log2);   // finite: column 0 is always valid
             float ps = 0.f;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                t[e] = fast_exp2(t[e] - m_new);
+                t[e] = fast_exp2(fmaf(t[e], p.scale_log2, -m_new));
                 ps += t[e];
             }
-            l_run[hf] = l_run[hf] * alpha + ps;
-            m_run[hf] = m_new;
+            // the accumulators are rescaled only when some row of the warp raised its maximum
+            // (always on the first block, rarely later)
+            if (__any_sync(0xffffffffu, m_new > m_run[hf])) {
+                const float alpha = fast_exp2(m_run[hf] - m_new);  // 0 on the first block
+                l_run[hf] = l_run[hf] * alpha + ps;
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                o[i][hf * 2 + 0] *= alpha;
-                o[i][hf * 2 + 1] *= alpha;
+                for (int i = 0; i < 16; ++i) {
+                    o[i][hf * 2 + 0] *= alpha;
+                    o[i][hf * 2 + 1] *= alpha;
+                }
+            } else {
+                l_run[hf] += ps;
             }
+            m_run[hf] = m_new;
             pa[hf] = pack_bf16(t[0], t[1]);          // tokens 0..7 of the block  (k low)
             pa[2 + hf] = pack_bf16(t[2], t[3]);      // tokens 8..15              (k high)
         }
