@@ -80,9 +80,12 @@ def test_whole_stack_step_with_mixed_layers(same_nr):
     hist = [[inputs.qkv_bf16(w, l, b, 0, lens[b]) for b in range(B)] for l in range(L)]
     dec = [[[inputs.qkv_bf16(w, l, b, lens[b] + i, 1) for b in range(B)] for l in range(L)] for i in range(steps)]
     results, stores = {}, {}
-    for mode in (0, 3):
-        cache = make(L, B, Hq, Hkv, S, W, [0] * L, [n + steps + 4 for n in lens], kvk=kvk, max_new=8192)
-        cache.tune("decode_overlap", mode)
+    # the third run keeps the retrieval rows in 128-token pages (one page per retrieval head and block)
+    pool = int(kvk.sum()) * sum((n + steps + 127) // 128 for n in lens)
+    for mode in (0, 3, "paged"):
+        cache = make(L, B, Hq, Hkv, S, W, [0] * L, [n + steps + 4 for n in lens], kvk=kvk, max_new=8192,
+                     pool_pages=pool if mode == "paged" else 0)
+        cache.tune("decode_overlap", 3 if mode == "paged" else mode)
         for l in range(L):
             k = np.concatenate([hist[l][b][1] for b in range(B)])
             v = np.concatenate([hist[l][b][2] for b in range(B)])
@@ -107,9 +110,11 @@ def test_whole_stack_step_with_mixed_layers(same_nr):
                         if (kvk[l] == (kind == binding.KIND_RETRIEVAL)).any()]
         cache.close()
     assert np.array_equal(results[0], results[3])
-    for a, b_ in zip(stores[0], stores[3]):
-        for x, y in zip(a, b_):
-            assert np.array_equal(np.asarray(x), np.asarray(y))
+    assert np.array_equal(results[0], results["paged"])
+    for other in (3, "paged"):
+        for a, b_ in zip(stores[0], stores[other]):
+            for x, y in zip(a, b_):
+                assert np.array_equal(np.asarray(x), np.asarray(y))
     scale = 1 / np.sqrt(D)
     for l in range(L):
         for b in range(B):
