@@ -252,12 +252,37 @@ def run_ours(args, w):
             # overlap from layer to layer) are sampled sparsely
             binding.profile_enable(args.profile_period * 64)
         lc = binding.launch_count()
-        for _ in range(steps_dec):
-            cache.decode_step_all(dq, dk, dv, dout)
+        extra = 0
+        if args.graph:
+            # the decode step captured into a CUDA graph and replayed; re-captured every args.graph
+            # steps so that the frozen split plan stays close to the growing stores.  Capture,
+            # instantiation and the length read-back are inside the timed region.
+            binding.profile_enable(0)          # no tracer events inside a capture
+            done = 0
+            while done < steps_dec:
+                n = min(args.graph, steps_dec - done)
+                cache.reserve(n)
+                g = torch.cuda.CUDAGraph()
+                lc0 = binding.launch_count()
+                with torch.cuda.stream(side):
+                    g.capture_begin()
+                    cache.decode_step_all(dq, dk, dv, dout)
+                    g.capture_end()
+                per_replay = binding.launch_count() - lc0
+                for _ in range(n):
+                    g.replay()
+                cache.sync_len()
+                extra += per_replay * (n - 1)   # the capture counted one step's launches and ran none
+                done += n
+        else:
+            for _ in range(steps_dec):
+                cache.decode_step_all(dq, dk, dv, dout)
         marks[2].record()
-        marks.append(binding.launch_count() - lc)
+        marks.append(binding.launch_count() - lc + extra)
+        marks.append(extra)
         return marks
 
+    side = torch.cuda.Stream(device=dev) if args.graph else None
     if not C:
         prefill_stores_ragged()
 
@@ -278,6 +303,7 @@ def run_ours(args, w):
     if world > 1:
         dist.barrier()
     launches = binding.launch_count() - launches0
+    launches += sum(m[4] for m in all_marks)     # graph replays are not seen by the library's counter
     clocks = sampler.stop() if sampler else None
     binding.profile_enable(0)
     prof = binding.profile_read(reset=True)
@@ -389,7 +415,7 @@ def run_ours(args, w):
     line = {"metric": METRIC, "value": us_per_token, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
             "ms_per_step": total_ms / K, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": w.name + ("+mixed" if args.mixed else "") + ("+paged" if args.paged else ""), "layers": L, "batch": B,
+            "config": {"workload": w.name + ("+mixed" if args.mixed else "") + ("+paged" if args.paged else "") + (f"+graph{args.graph}" if args.graph else ""), "layers": L, "batch": B,
                        "q_heads": Hq, "kv_heads": Hkv, "head_dim": D, "sink": w.sink, "recent": w.recent,
                        "retrieval_layers": nR_layers, "prefill_len": w.prefill_len, "prefill_chunk": C,
                        "decode_steps": steps_dec, "decode_overlap": args.decode_overlap if args.decode_overlap >= 0 else 3,
@@ -463,6 +489,8 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--paged", action="store_true",
                     help="retrieval stores in 128-token pages from a shared pool (a variant, not the default)")
+    ap.add_argument("--graph", type=int, default=0, metavar="N",
+                    help="replay the decode step from a CUDA graph, re-captured every N steps (0: plain launches)")
     ap.add_argument("--decode-steps", type=int, default=-1, help="override the workload's decode steps")
     ap.add_argument("--mixed", action="store_true", help="mixed-head (two-pass) arm of the comparison")
     ap.add_argument("--share-inputs", action="store_true", help="one set of prefill tensors for all layers")

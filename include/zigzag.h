@@ -113,6 +113,20 @@ int zz_cache_create_paged(const zz_config_t* cfg, int32_t pool_pages, void* d_ar
                           void* d_workspace, size_t workspace_bytes, zz_cache_t** out);
 /* Pages of the pool and pages free now (both 0 for a cache with contiguous stores). */
 int zz_cache_pages(const zz_cache_t* cache, int32_t* total, int32_t* free_now);
+/* Replaying decode steps from a CUDA graph.  zz_decode_step / zz_decode_step_all may be captured
+ * into a graph (they only launch kernels); a replay repeats the launch plan of the capture, the
+ * kernels take the lengths from device memory, and the last split of each sequence absorbs the
+ * tokens added since the capture (re-capture every few hundred steps to keep the splits even).
+ * The host does not see replays, so: (1) before capturing, call zz_cache_reserve with the number
+ * of steps that will be replayed: it checks the capacities and, for a paged cache, takes the
+ * pages now (ZZ_ERR_CAPACITY, nothing changed, if they do not fit); (2) after the replays, call
+ * zz_cache_sync_len, which reads the device lengths back into the host mirror (it synchronises
+ * the stream).  A replay that runs out of room anyway is refused on the device: the kernels of
+ * that sequence's retrieval layers store and write nothing and zz_get_last_status returns
+ * ZZ_ERR_CAPACITY (the sequence is then inconsistent across layers: reset it).  The capture call
+ * itself counts as one step in the host mirror but executes nothing. */
+int zz_cache_reserve(zz_cache_t* cache, int32_t extra_tokens, void* stream);
+int zz_cache_sync_len(zz_cache_t* cache, void* stream);
 /* Frees the host handle (device memory stays the caller's). */
 int zz_cache_destroy(zz_cache_t* cache);
 /* Forgets the tokens of sequence `seq` (-1: all sequences) in every layer. */

@@ -65,6 +65,8 @@ SYMBOLS = {
     "zz_cache_query_paged": (_i32, [_cfgp, _i32, ctypes.POINTER(_sz), ctypes.POINTER(_sz)]),
     "zz_cache_create_paged": (_i32, [_cfgp, _i32, _vp, _sz, _vp, _sz, ctypes.POINTER(_vp)]),
     "zz_cache_pages": (_i32, [_vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]),
+    "zz_cache_reserve": (_i32, [_vp, _i32, _vp]),
+    "zz_cache_sync_len": (_i32, [_vp, _vp]),
     "zz_cache_destroy": (_i32, [_vp]),
     "zz_cache_reset": (_i32, [_vp, _i32, _vp]),
     "zz_cache_len": (_i32, [_vp, _i32, _i32, ctypes.POINTER(ctypes.c_int32)]),
@@ -248,6 +250,14 @@ class ZigzagCache:
         t, f = ctypes.c_int32(0), ctypes.c_int32(0)
         _check(self._lib.zz_cache_pages(self._h, ctypes.byref(t), ctypes.byref(f)), "zz_cache_pages")
         return int(t.value), int(f.value)
+
+    def reserve(self, extra_tokens: int, stream=None) -> None:
+        """Room (and, for a paged cache, pages) for `extra_tokens` more tokens in every sequence."""
+        _check(self._lib.zz_cache_reserve(self._h, int(extra_tokens), _stream_ptr(stream)), "zz_cache_reserve")
+
+    def sync_len(self, stream=None) -> None:
+        """Host mirror of the lengths := device lengths (after decode steps replayed from a CUDA graph)."""
+        _check(self._lib.zz_cache_sync_len(self._h, _stream_ptr(stream)), "zz_cache_sync_len")
 
     def tune(self, key: str, value: int) -> None:
         _check(self._lib.zz_tune(self._h, key.encode(), int(value)), "zz_tune")

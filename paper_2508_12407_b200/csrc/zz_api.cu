@@ -629,7 +629,7 @@ static int create_impl(const zz_config_t* cfg, long long pool_pages, void* d_are
     c->pool_pages = (int)pool_pages;
     c->table_dirty = false;
     if (c->paged) {
-        c->h_table.assign((size_t)c->lay.table_entries, 0);
+        c->h_table.assign((size_t)c->lay.table_entries, -1);
         c->pages_of.assign((size_t)c->L * c->B, 0);
         c->free_pages.resize((size_t)pool_pages);
         for (long long i = 0; i < pool_pages; ++i) c->free_pages[(size_t)i] = (int)(pool_pages - 1 - i);  // page 0 on top
@@ -678,6 +678,8 @@ static int create_impl(const zz_config_t* cfg, long long pool_pages, void* d_are
     if (e == cudaSuccess) e = cudaMemset(c->arena, 0, c->lay.arena_bytes);
     if (e == cudaSuccess) e = cudaMemset(c->work, 0, c->lay.off_part_ml);
     if (e == cudaSuccess) e = cudaMemset(c->work + c->lay.off_pos, 0xff, (size_t)c->L * c->B * c->ring * sizeof(int));
+    if (e == cudaSuccess && c->lay.table_entries > 0)     // no page anywhere yet
+        e = cudaMemset(c->work + c->lay.off_table, 0xff, (size_t)c->lay.table_entries * sizeof(int));
     if (e == cudaSuccess)
         e = cudaMemcpy(c->work + c->lay.off_desc, c->desc.data(), c->desc.size() * sizeof(SeqDesc),
                        cudaMemcpyHostToDevice);
@@ -709,6 +711,9 @@ int zz_cache_reset(zz_cache_t* c, int seq, void* stream) {
     c->last_nowait = false;
     if (zz::launch_reset(c->d_len(0), c->d_pos(0), c->L, c->B, c->ring, seq, st) != cudaSuccess)
         return ZZ_ERR_CUDA;
+    zz::TableUpdate u;
+    u.n = 0;
+    bool ok = true;
     for (int l = 0; l < c->L; ++l)
         for (int b = 0; b < c->B; ++b)
             if (seq < 0 || seq == b) {
@@ -716,18 +721,53 @@ int zz_cache_reset(zz_cache_t* c, int seq, void* stream) {
                 c->len[lb] = 0;
                 if (c->paged) {
                     // the sequence's pages go back to the pool (work already in the stream that reads
-                    // them is ordered before whatever writes them next on the same stream)
+                    // them is ordered before whatever writes them next on the same stream); their
+                    // table entries read "no page" again
                     const int n = c->pages_of[lb] * c->nR[l];
-                    for (int i = 0; i < n; ++i) c->free_pages.push_back(c->h_table[c->desc[lb].tbl + i]);
+                    for (int i = 0; i < n; ++i) {
+                        const int idx = c->desc[lb].tbl + i;
+                        c->free_pages.push_back(c->h_table[idx]);
+                        c->h_table[idx] = -1;
+                        u.idx[u.n] = idx;
+                        u.val[u.n] = -1;
+                        if (++u.n == 480) {
+                            ok = ok && zz::launch_table_update(c->d_table(), u, st) == cudaSuccess;
+                            u.n = 0;
+                        }
+                    }
                     c->pages_of[lb] = 0;
                 }
             }
-    return ZZ_OK;
+    if (u.n > 0) ok = ok && zz::launch_table_update(c->d_table(), u, st) == cudaSuccess;
+    return ok ? ZZ_OK : ZZ_ERR_CUDA;
 }
 
 int zz_cache_len(const zz_cache_t* c, int layer, int seq, int32_t* len) {
     if (bad_layer(c, layer) || seq < 0 || seq >= c->B || !len) return ZZ_ERR_INVALID_ARG;
     *len = c->len[(size_t)layer * c->B + seq];
+    return ZZ_OK;
+}
+
+int zz_cache_reserve(zz_cache_t* c, int32_t extra_tokens, void* stream) {
+    if (!c || extra_tokens < 0) return ZZ_ERR_INVALID_ARG;
+    for (int l = 0; l < c->L; ++l)
+        for (int b = 0; b < c->B; ++b) {
+            const long long nl = (long long)c->len[(size_t)l * c->B + b] + extra_tokens;
+            if (nl > 0x7fffffffLL || (c->nR[l] > 0 && nl > c->cap[b])) return ZZ_ERR_CAPACITY;
+        }
+    int32_t add[ZZ_MAX_BATCH];
+    for (int b = 0; b < c->B; ++b) add[b] = extra_tokens;
+    return reserve_pages(c, 0, c->L, add, static_cast<cudaStream_t>(stream));
+}
+
+int zz_cache_sync_len(zz_cache_t* c, void* stream) {
+    if (!c) return ZZ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    std::vector<int> dev(c->len.size());
+    if (cudaMemcpyAsync(dev.data(), c->d_len(0), dev.size() * sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return ZZ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ZZ_ERR_CUDA;
+    c->len = dev;
     return ZZ_OK;
 }
 

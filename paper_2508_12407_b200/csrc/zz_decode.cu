@@ -174,6 +174,18 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     int new_slot = -1;
     const __nv_bfloat16* knew = nullptr;
     const __nv_bfloat16* vnew = nullptr;
+    if (fused && p.kind == ZZ_KIND_RETRIEVAL) {
+        // Room for the appended row?  The host checks this before it launches; a launch replayed
+        // from a CUDA graph has no host check, so the kernel refuses by itself: every CTA of the
+        // sequence sees the same length and returns before it touches the store, the scratch or the
+        // output, and the status word tells the host.
+        bool room = len_old < sd.cap;
+        if (paged && room) room = tbl[(len_old >> 7) * p.Hg] >= 0;
+        if (!room) {
+            if (threadIdx.x == 0) atomicCAS(p.status, 0, ZZ_ERR_CAPACITY);
+            return;
+        }
+    }
     if (fused) {
         const int t = len_old;
         new_slot = (p.kind == ZZ_KIND_RETRIEVAL || t < p.S) ? t : p.S + ((t - p.S) % p.W);
