@@ -38,8 +38,9 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int sr
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes)
                  : "memory");
 }
-__device__ __forceinline__ void cp_async16_full(uint32_t dst, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
+__device__ __forceinline__ void cp_async16_full(uint32_t dst, const void* src, uint64_t policy) {
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "l"(policy)
+                 : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
@@ -87,7 +88,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // row comes from the caller's k_new/v_new instead of the store.
 __device__ __forceinline__ void load_block(uint32_t stage_k, uint32_t stage_v, const __nv_bfloat16* kbase,
                                            const __nv_bfloat16* vbase, int tok0, int tok_end, int lane,
-                                           int new_slot, const __nv_bfloat16* knew, const __nv_bfloat16* vnew) {
+                                           int new_slot, const __nv_bfloat16* knew, const __nv_bfloat16* vnew,
+                                           uint64_t policy) {
     if (tok0 + kBlk <= tok_end && (new_slot < tok0 || new_slot >= tok0 + kBlk)) {
         // Whole block from the store (all but the edge blocks of a range): one pointer per lane, every
         // further address a constant away.  Row r = 2*it + r0 swizzles with (r & 7) = 2*(it & 3) + r0,
@@ -100,8 +102,8 @@ __device__ __forceinline__ void load_block(uint32_t stage_k, uint32_t stage_v, c
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
             const uint32_t so = (so0 ^ ((it & 3) << 5)) + it * 2 * kRowBytes;
-            cp_async16_full(stage_k + so, kp + it * 2 * kD);
-            cp_async16_full(stage_v + so, vp + it * 2 * kD);
+            cp_async16_full(stage_k + so, kp + it * 2 * kD, policy);
+            cp_async16_full(stage_v + so, vp + it * 2 * kD, policy);
         }
         return;
     }
@@ -238,6 +240,14 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     float l_run[2] = {0.f, 0.f};
 
     const uint32_t wbase = smem_u32(smem) + warp * kWarpSmem;
+    // L2 policy of the K/V loads: a retrieval store is streamed once per step and should not push
+    // anything out of the L2 (evict first); the rings of the streaming layers are read again by the
+    // next step and together fit the L2 (evict last)
+    uint64_t l2_policy;
+    if (p.kind == ZZ_KIND_RETRIEVAL)
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(l2_policy));
+    else
+        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(l2_policy));
 
     // Paged store: lane i holds the page of token block pg0 + i (32 pages = 4096 tokens); a block's
     // page is a shuffle away, the window is reloaded when the warp walks past it.  Blocks start at
@@ -264,7 +274,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
             const int tok0 = s0 + (warp + s * kWarps) * kBlk;
             const long long po = page_off(tok0);
             load_block(wbase + s * 2 * kStageBytes, wbase + s * 2 * kStageBytes + kStageBytes, kbase + po, vbase + po,
-                       tok0, s1, lane, new_slot, knew, vnew);
+                       tok0, s1, lane, new_slot, knew, vnew, l2_policy);
         }
         cp_async_commit();
     }
@@ -277,7 +287,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
                 const int tok0 = s0 + (warp + nx * kWarps) * kBlk;
                 const long long po = page_off(tok0);
                 load_block(wbase + st * 2 * kStageBytes, wbase + st * 2 * kStageBytes + kStageBytes, kbase + po,
-                           vbase + po, tok0, s1, lane, new_slot, knew, vnew);
+                           vbase + po, tok0, s1, lane, new_slot, knew, vnew, l2_policy);
             }
             cp_async_commit();
         }
