@@ -140,8 +140,10 @@ int zz_cache_len(const zz_cache_t* cache, int layer, int seq, int32_t* len);
  * total_tokens * kv_heads <= SMs * value below which it is used; multiple of 16, default
  * 384; 0 disables the short-store plan); "decode_overlap" (how the layers
  * of zz_decode_step_all are launched.  3, the default: all exclusive retrieval layers in one
- * launch and all exclusive streaming layers in another (possible when no layer is mixed and all
- * layers hold equally long sequences; otherwise as 2); 2: one launch per layer, programmatic
+ * launch and all exclusive streaming layers in another; the mixed layers, if they all have the
+ * same number of retrieval heads, in one launch per pass plus one head-regrouping copy before and
+ * one after (possible when all layers hold equally long sequences; otherwise as 2, with the
+ * four launches of a mixed layer in plain order); 2: one launch per layer, programmatic
  * dependent launch and no wait between layers -- they share no scratch, so a layer's kernel fills
  * the SMs the previous one leaves idle; 1: the same, but each kernel waits for the previous one
  * before it merges; 0: plain stream order); "decode_multi_waves" (default 8: a grid over n layers
@@ -177,9 +179,10 @@ int zz_decode_attn(zz_cache_t* cache, int layer, const void* d_q, void* d_out, v
 int zz_decode_step(zz_cache_t* cache, int layer, const void* d_q, const void* d_k,
                    const void* d_v, void* d_out, void* stream);
 
-/* One decode step of the whole stack: zz_decode_step for layers 0 .. n_layers-1 in order.
- * d_q/d_out: [n_layers, batch, n_q_heads, 128]; d_k/d_v: [n_layers, batch, n_kv_heads, 128].
- * Capacity is validated for every layer before anything is launched. */
+/* One decode step of the whole stack: the result of zz_decode_step for every layer, with the
+ * q/k/v of all layers given up front (d_q/d_out: [n_layers, batch, n_q_heads, 128]; d_k/d_v:
+ * [n_layers, batch, n_kv_heads, 128]), which lets the layers share launches (see "decode_overlap"
+ * under zz_tune).  Capacity is validated for every layer before anything is launched. */
 int zz_decode_step_all(zz_cache_t* cache, const void* d_q, const void* d_k, const void* d_v,
                        void* d_out, void* stream);
 
