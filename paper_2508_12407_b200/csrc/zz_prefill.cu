@@ -36,7 +36,7 @@ constexpr int kStages = 4;                  // K/V tiles held at once: two pair 
 constexpr int kPairs = 2;                   // one full / empty barrier per pair: what an iteration uses, it uses together
 constexpr int kThreads = 384;                // three warpgroups: softmax tile 0, softmax tile 1, TMA + MMA
 constexpr int kWarpTma = 8, kWarpMma = 9;
-constexpr int kRegsSoftmax = 208, kRegsAux = 88;   // 208 * 256 + 88 * 128 <= 65536 registers
+constexpr int kRegsSoftmax = 200, kRegsAux = 104;  // 200 * 256 + 104 * 128 = 64512 registers, what the launch allocates (168 * 384)
 constexpr int kEpiBytes = 8 * 4096;          // output staging: 16 rows of 256 B per softmax warp
 constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + kEpiBytes + 1024;
 constexpr uint32_t kMaxPolls = 1u << 22;
