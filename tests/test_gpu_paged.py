@@ -11,6 +11,7 @@ from test_gpu_prefill import run_prefill
 from zz_testlib import OracleSeq, assert_close, to_bits, to_dev
 
 pytestmark = pytest.mark.gpu
+D = 128
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -151,3 +152,36 @@ def test_paged_export_import_roundtrip():
     assert np.array_equal(to_bits(oa), to_bits(ob))
     a.close()
     b.close()
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_million_token_store_maximum_splits(paged):
+    """One KV head with a million tokens: the split plan runs into its limit of 120 splits, every
+    CTA's range spans more than 32 pages (the paged kernel reloads its window of page ids) and a
+    warp walks ~2000 tokens.  Decode rows against the oracle over the full history."""
+    import oracle
+    Hq, Hkv, S, W = 4, 1, 4, 12
+    n, steps = 1_000_000, 2
+    cap = n + steps
+    pool = (cap + 127) // 128 if paged else 0
+    cache = make(1, 1, Hq, Hkv, S, W, [1], [cap], max_new=65536, pool_pages=pool)
+    hk = np.empty((cap, Hkv, D), np.uint16)
+    hv = np.empty((cap, Hkv, D), np.uint16)
+    done = 0
+    while done < n:
+        c = min(65536, n - done)
+        hk[done:done + c] = inputs.normal_bf16((c, Hkv, D), 4321, 1, done)
+        hv[done:done + c] = inputs.normal_bf16((c, Hkv, D), 4321, 2, done)
+        cache.kv_append(0, to_dev(hk[done:done + c]), to_dev(hv[done:done + c]), [c])
+        done += c
+    for i in range(steps):
+        q = inputs.normal_bf16((1, Hq, D), 4321, 3, i)
+        hk[n + i] = inputs.normal_bf16((1, Hkv, D), 4321, 4, i)[0]
+        hv[n + i] = inputs.normal_bf16((1, Hkv, D), 4321, 5, i)[0]
+        dq = to_dev(q)
+        out = dq.new_zeros(dq.shape)
+        cache.decode_step(0, dq, to_dev(hk[n + i:n + i + 1]), to_dev(hv[n + i:n + i + 1]), out)
+        want = oracle.attn_rows(q, [n + i], hk[:n + i + 1], hv[:n + i + 1], [1], S, W, 1 / np.sqrt(D))
+        assert_close(to_bits(out), want, f"step {i}")
+    assert cache.last_status() == 0 and cache.len(0, 0) == n + steps
+    cache.close()
