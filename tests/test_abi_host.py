@@ -95,3 +95,39 @@ def test_null_arguments(lib):
     assert lib.zz_prefill_attn(None, 0, None, None, None, None, None, None) == binding.ZZ_ERR_INVALID_ARG
     assert lib.zz_get_last_status(None, None) == binding.ZZ_ERR_INVALID_ARG
     assert lib.zz_stage_bytes(None, 5) == 0
+
+
+def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
+    # no fallback of any kind: a missing extension is an ImportError that says how to build it
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "libzigzag_b200.so"))
+    with pytest.raises(ImportError) as e:
+        binding.load()
+    assert "build" in str(e.value)
+
+
+def test_no_product_module_imports_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2508_12407_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f), errors="ignore").read()
+                assert not re.search(r"^\s*(import|from)\s+oracle\b", text, flags=re.M), f
+                assert "zz_oracle" not in text, f
+
+
+def test_paged_query_sizes_pool_and_table(lib):
+    cfg = make_cfg(L=3, B=2, kinds=[1, 0, 1], cap=[1000, 300], Hq=8, Hkv=2, S=16, W=48)
+    rc0, a0, w0 = query(lib, cfg)
+    assert rc0 == 0
+    a, w = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    assert lib.zz_cache_query_paged(ctypes.byref(cfg), 0, ctypes.byref(a), ctypes.byref(w)) == binding.ZZ_ERR_INVALID_ARG
+    pool = 40
+    assert lib.zz_cache_query_paged(ctypes.byref(cfg), pool, ctypes.byref(a), ctypes.byref(w)) == 0
+    # arena: the contiguous retrieval stores (2 layers x 2 heads x (1000 + 300) slots x K and V) are
+    # replaced by the pool of 64 KB pages; the rings stay
+    contiguous = 2 * 2 * (1000 + 300) * 128 * 2 * 2
+    assert abs((a0 - contiguous + pool * 65536) - a.value) <= 512
+    # workspace: + the page table, 2 retrieval layers x 2 heads x (ceil(1000/128) + ceil(300/128)) entries
+    entries = 2 * 2 * (8 + 3)
+    assert 0 <= (w.value - w0) - entries * 4 <= 512
