@@ -564,7 +564,6 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
             const TilePlan plan = it.plan;
             const int r = quarter * 32 + lane;          // query row inside the tile
             const int rr = r0 + r;                      // row inside the chunk
-            const int* pos = p.pos + (long long)b * p.ring;
             float m_used = -INFINITY, l_run = 0.f;
             for (int j = 0; j < n_tiles; ++j) {
                 bool is_chunk;
@@ -601,21 +600,22 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
 #pragma unroll
                         for (int w = 0; w < 4; ++w) vis[w] = range_bits(0, lim - 1, 32 * w);
                     } else if (!is_chunk) {
+                        // Ring slots visible to the query at position tq: the sinks, and the stored tokens
+                        // t >= tq - W + 1.  After P appended tokens the ring holds tokens max(S, P - W) .. P - 1
+                        // at slots S + ((t - S) mod W), so a run of consecutive tokens is a run of consecutive
+                        // slots that wraps at most once: three slot ranges instead of a look-up per column.
                         const int tq = P + rr;
+                        const int n_sink = min(p.S, P);
+                        const int lo_t = max(max(p.S, P - p.W), tq - p.W + 1);   // first visible stored non-sink token
+                        const int n_rec = max(P - lo_t, 0);
+                        const int a = p.S + (lo_t - p.S) % p.W;                  // its slot
+                        const int e1 = min(a + n_rec, p.ring);                   // end of the run before the wrap
+                        const int wrap = a + n_rec - e1;                         // slots of the run after the wrap
 #pragma unroll
                         for (int w = 0; w < 4; ++w) {
-                            uint32_t m = 0;
-#pragma unroll 4
-                            for (int i = 0; i < 32; ++i) {
-                                const int idx = start + 32 * w + i;
-                                bool ok = idx < plan.n_occ;
-                                if (ok) {
-                                    const int pp = pos[idx];
-                                    ok = (pp < p.S) || (tq - pp < p.W);
-                                }
-                                m |= (ok ? 1u : 0u) << i;
-                            }
-                            vis[w] = m;
+                            const int base = start + 32 * w;
+                            vis[w] = range_bits(0, n_sink - 1, base) |
+                                     (n_rec > 0 ? range_bits(a, e1 - 1, base) | range_bits(p.S, p.S + wrap - 1, base) : 0u);
                         }
                     } else {
                         const int c_hi = rr - start;                      // causal
