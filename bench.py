@@ -66,13 +66,23 @@ class ClockSampler:
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_index: int):
+        # started before the warm-up (nvidia-smi takes a few hundred ms to deliver its first sample);
+        # only what it writes after mark() counts
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         self.p = None
+        self.skip = 0
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
                                        "-i", str(gpu_index), "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
+
+    def mark(self):
+        """The timed region starts now: earlier samples are dropped."""
+        try:
+            self.skip = os.path.getsize(self.f.name)
+        except OSError:
+            self.skip = 0
 
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
@@ -84,9 +94,9 @@ class ClockSampler:
         except Exception:
             self.p.kill()
         self.f.flush()
-        self.f.seek(0)
+        self.f.seek(self.skip)
         sm, mx, reasons = [], [], set()
-        for line in self.f.read().splitlines():
+        for line in self.f.read().splitlines()[1 if self.skip else 0:]:   # the first line after mark() may be cut
             parts = [x.strip() for x in line.split(",")]
             if len(parts) < 9:
                 continue
@@ -286,12 +296,14 @@ def run_ours(args, w):
     if not C:
         prefill_stores_ragged()
 
+    sampler = ClockSampler(local) if rank == 0 else None
     for _ in range(args.warmup):
         step(False)
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
-    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.mark()
     binding.profile_read(reset=True)
     launches0 = binding.launch_count()
     t0, t1 = ev(), ev()
