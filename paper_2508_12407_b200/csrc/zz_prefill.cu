@@ -639,8 +639,43 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                 // long as its two MMAs; on tiles without masked (-inf) entries every kPolyEvery-th
                 // pair is therefore evaluated by a polynomial on the FMA pipe instead.
                 float psum = 0.f;
+                // The common tile (nothing masked, not the item's first) runs straight through: every
+                // uniform branch between "S is here" and "P is there" costs tens of cycles on the path
+                // that the tensor pipe waits for.  If the maximum did move, the general loop below redoes it.
+                bool done = false;
+                if (!tile_masked && j > 0) {
+                    // (a row that has seen nothing yet has m_used = -inf: any finite score then counts as a
+                    // move of the maximum, and the general loop takes over)
+                    const float msub = (m_used == -INFINITY) ? 0.f : m_used;
+                    const float2 sc2 = make_float2(sc, sc), nm2 = make_float2(-msub, -msub);
+                    float2 ps2 = make_float2(0.f, 0.f);
+                    float mc[4];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t pk[16];
+                        float a = s[c * 32];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const float s0 = s[c * 32 + 2 * i], s1 = s[c * 32 + 2 * i + 1];
+                            a = max3(a, s0, s1);
+                            const float2 x = fma2(make_float2(s0, s1), sc2, nm2);
+                            const float2 e = ((i % kPolyEvery) == kPolyEvery - 1)
+                                                 ? exp2_poly2(x)
+                                                 : make_float2(fast_exp2(x.x), fast_exp2(x.y));
+                            ps2 = add2(ps2, e);
+                            pk[i] = pack_bf16(e.x, e.y);
+                        }
+                        mc[c] = a;
+                        tmem_st16(t_s + c * 16, pk);
+                    }
+                    const float mx = fmaxf(max3(mc[0], mc[1], mc[2]), mc[3]) * sc;
+                    if (!__any_sync(0xffffffffu, mx > m_used + kRescaleThreshold)) {
+                        psum = ps2.x + ps2.y;
+                        done = true;
+                    }
+                }
 #pragma unroll 1
-                for (int attempt = 0; attempt < 2; ++attempt) {
+                for (int attempt = done ? 2 : 0; attempt < 2; ++attempt) {
                     const bool do_exp = (attempt == 1) || (j > 0);
                     float mc[4];
                     if (do_exp) {
