@@ -14,6 +14,12 @@
 // the split merge, so there is no second launch.
 //
 // The roofline of this kernel is HBM bandwidth: 2 * 128 * 2 bytes per token and KV head.
+//
+// Also here: the append of the step's new token fused into the launch (its row is taken from the
+// caller's tensors, stored in its slot and attended to; the kernel refuses by itself when a
+// retrieval store has no room, for launches replayed from a CUDA graph), a grid over several
+// layers (blockIdx.y), paged retrieval stores (separate instantiations), L2 policy hints on the
+// K/V loads, and the programmatic-dependent-launch hooks that let consecutive launches overlap.
 #include <cstring>
 
 #include "zz_common.cuh"
