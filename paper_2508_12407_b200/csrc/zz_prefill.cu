@@ -5,11 +5,13 @@
 // diagonal (causal flash attention); a streaming head visits only the tiles that can hold
 // visible keys -- the sink tiles and the local band -- and applies the token-exact
 // visibility rule inside them (block sparsity is an execution strategy, not the mask).
-// Keys come from two places: the store as it stood before the call (append-only rows or
-// ring slots, positions from pos[]) and the new chunk itself.
+// Keys come from two places: the store as it stood before the call (append-only rows, contiguous
+// or in 128-token pages; or ring slots, whose tokens follow from the length) and the new chunk.
 //
-// CTA = one 128-token query tile x two query heads of the same KV head, so each K/V tile is
-// fetched once for two score tiles and the two tiles ping-pong on the tensor pipe:
+// Work item = one 128-token query tile x two query heads of the same KV head, so each K/V tile is
+// fetched once for two score tiles and the two tiles ping-pong on the tensor pipe.  A CTA works
+// through a static share of the items (one CTA per SM; one item per CTA when a launch has no more
+// items than SMs):
 //   warps 0-3   softmax / correction / epilogue of tile 0 (one thread per query row)
 //   warps 4-7   the same for tile 1
 //   warp 8      TMA producer (one elected lane)
