@@ -111,7 +111,7 @@ struct GatherParams {
 struct PrefillParams {
     const SeqDesc* desc;     // [B] of this layer
     const int* len;          // [B] device lengths (tokens already in the store)
-    const int* pos;          // [B][ring] ring positions of this layer
+    const int* pos;          // [B][ring] ring positions of this layer (not read: which token a slot holds follows from len)
     __nv_bfloat16* out;      // row of packed token i, head h at out + i*tok_stride + (q_head0+h)*128
     long long tok_stride;    // n_q_heads * 128
     const int* page_table;   // nullptr: contiguous retrieval stores
