@@ -451,9 +451,12 @@ def run_ours(args, w):
 
     # ---- end to end through host buffers (pinned), one step ---------------------------------
     if rank == 0 and not args.no_e2e and steps_dec:
-        hq = torch.empty(L, B, Hq, D, dtype=torch.bfloat16).pin_memory()
-        hk = torch.empty(L, B, Hkv, D, dtype=torch.bfloat16).pin_memory()
-        hv = torch.empty(L, B, Hkv, D, dtype=torch.bfloat16).pin_memory()
+        # q, k and v of a step back to back in one pinned buffer: the library then sends them in one copy
+        nq, nk = L * B * Hq * D, L * B * Hkv * D
+        hbuf = torch.empty(nq + 2 * nk, dtype=torch.bfloat16).pin_memory()
+        hq = hbuf[:nq].view(L, B, Hq, D)
+        hk = hbuf[nq:nq + nk].view(L, B, Hkv, D)
+        hv = hbuf[nq + nk:].view(L, B, Hkv, D)
         ho = torch.empty(L, B, Hq, D, dtype=torch.bfloat16).pin_memory()
         hq.copy_(dq); hk.copy_(dk); hv.copy_(dv)
         stage = torch.empty(cache.stage_bytes(L * B), dtype=torch.uint8, device=dev)

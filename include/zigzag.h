@@ -196,7 +196,8 @@ int zz_decode_step_host(zz_cache_t* cache, int layer, const void* h_q, const voi
                         void* stream);
 /* zz_decode_step_all fed from HOST memory: h_q/h_out [n_layers, batch, n_q_heads, 128], h_k/h_v
  * [n_layers, batch, n_kv_heads, 128]; d_stage holds at least
- * zz_stage_bytes(cache, n_layers * batch) bytes. */
+ * zz_stage_bytes(cache, n_layers * batch) bytes.  When h_q, h_k and h_v lie back to back in host
+ * memory (in that order) they travel in one copy. */
 int zz_decode_step_all_host(zz_cache_t* cache, const void* h_q, const void* h_k, const void* h_v,
                             void* h_out, void* d_stage, size_t stage_bytes, void* stream);
 int zz_prefill_host(zz_cache_t* cache, int layer, const void* h_q, const void* h_k,

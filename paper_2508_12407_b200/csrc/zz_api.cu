@@ -1120,9 +1120,16 @@ int zz_decode_step_all_host(zz_cache_t* c, const void* h_q, const void* h_k, con
     const size_t qb = align_up(qbytes), kb = align_up(kbytes);
     unsigned char* s = static_cast<unsigned char*>(d_stage);
     void* dq = s; void* dk = s + qb; void* dv = s + qb + kb; void* dout = s + qb + 2 * kb;
-    if (cudaMemcpyAsync(dq, h_q, qbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ZZ_ERR_CUDA;
-    if (cudaMemcpyAsync(dk, h_k, kbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ZZ_ERR_CUDA;
-    if (cudaMemcpyAsync(dv, h_v, kbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    const char* hq = static_cast<const char*>(h_q);
+    if (static_cast<const char*>(h_k) == hq + qbytes && static_cast<const char*>(h_v) == hq + qbytes + kbytes &&
+        qb == qbytes && kb == kbytes) {
+        // q, k and v lie back to back on the host (and so they do in the staging buffer): one copy
+        if (cudaMemcpyAsync(dq, h_q, qbytes + 2 * kbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    } else {
+        if (cudaMemcpyAsync(dq, h_q, qbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ZZ_ERR_CUDA;
+        if (cudaMemcpyAsync(dk, h_k, kbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ZZ_ERR_CUDA;
+        if (cudaMemcpyAsync(dv, h_v, kbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    }
     const int r = zz_decode_step_all(c, dq, dk, dv, dout, stream);
     if (r != ZZ_OK) return r;
     if (cudaMemcpyAsync(h_out, dout, qbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZZ_ERR_CUDA;

@@ -43,7 +43,7 @@ def test_host_entries_match_device_entries():
         torch.cuda.synchronize()
         assert np.array_equal(to_bits(out), to_bits(ho))
     # one decode step through the whole-stack host entry, one through the per-layer host entry
-    for step in range(2):
+    for step in range(3):
         qkv = [[inputs.qkv_bf16(w, l, b, C + step, 1) for b in range(B)] for l in range(L)]
         q = np.stack([np.concatenate([qkv[l][b][0] for b in range(B)]) for l in range(L)])
         k = np.stack([np.concatenate([qkv[l][b][1] for b in range(B)]) for l in range(L)])
@@ -55,6 +55,14 @@ def test_host_entries_match_device_entries():
         hq, hk, hv = _pinned(q), _pinned(k), _pinned(v)
         if step == 0:
             host_c.decode_step_all_host(hq, hk, hv, ho, stage)
+        elif step == 2:
+            # q, k, v back to back in one pinned buffer: the library sends them in one copy
+            buf = torch.empty(hq.numel() + hk.numel() + hv.numel(), dtype=hq.dtype).pin_memory()
+            nq, nk = hq.numel(), hk.numel()
+            bq, bk, bv = buf[:nq].view(hq.shape), buf[nq:nq + nk].view(hk.shape), buf[nq + nk:].view(hv.shape)
+            bq.copy_(hq); bk.copy_(hk); bv.copy_(hv)
+            assert bk.data_ptr() == bq.data_ptr() + nq * 2 and bv.data_ptr() == bk.data_ptr() + nk * 2
+            host_c.decode_step_all_host(bq, bk, bv, ho, stage)
         else:
             for l in range(L):
                 host_c.decode_step_host(l, hq[l], hk[l], hv[l], ho[l], stage)
