@@ -218,9 +218,21 @@ int zz_cache_export(zz_cache_t* cache, int layer, int seq, int kind, void* h_k, 
 int zz_cache_import(zz_cache_t* cache, int layer, int seq, int kind, const void* h_k,
                     const void* h_v, const int32_t* h_pos, int32_t len, void* stream);
 
-/* Reads (and clears) the device status word: ZZ_OK, or ZZ_ERR_TIMEOUT if a bounded wait
- * inside a kernel expired since the last read.  Synchronises the stream. */
+/* Reads (and clears) the device status word: ZZ_OK, ZZ_ERR_TIMEOUT if a bounded wait inside a
+ * kernel expired since the last read, ZZ_ERR_CAPACITY if a replayed decode step found a retrieval
+ * store full, ZZ_ERR_UNSUPPORTED if a decode launch was refused for a split plan beyond the
+ * kernel's limit.  Synchronises the stream. */
 int zz_get_last_status(zz_cache_t* cache, void* stream);
+
+/* Self-test of the failure path of the kernels' bounded waits (the paper has no counterpart).
+ * Every wait inside the kernels (on a shared-memory barrier that a copy or an MMA completes) gives
+ * up after a fixed number of probes, records ZZ_ERR_TIMEOUT in the status word and lets the
+ * kernel return, so a wait that can never end costs a status instead of a hung device.  This
+ * call launches one warp that runs that same wait on a barrier nothing ever completes, with the
+ * limit set to max_polls (1 .. 65536) and no copy or MMA in flight; it returns ZZ_OK once the
+ * kernel has given up and returned (it synchronises the stream), and the next
+ * zz_get_last_status then reports ZZ_ERR_TIMEOUT.  The device context stays usable. */
+int zz_selftest_wait_timeout(zz_cache_t* cache, int32_t max_polls, void* stream);
 
 /* Tracer (the paper has no counterpart; it reports per-token latencies only, Section 3.2).
  * zz_profile_enable(n): n = 0 switches it off; n >= 1 brackets every n-th launch of each
@@ -236,12 +248,15 @@ int zz_profile_read(int kind, int64_t* launches, double* total_ms, int reset);
  * is a deployment convenience, not part of the method).
  *
  * For callers that cannot allocate device memory -- a server that has given the whole device
- * to its own pool, a plug-in whose host forbids allocations after start-up, code that may run
- * while a stream is being captured -- and therefore cannot hand the library a workspace.  The
- * scratch the split-sequence decode kernel needs (partial outputs, their softmax statistics,
- * arrival counters, the device copy of the lengths) lives in a fixed array of about 2.1 MB
- * inside the library's device image; every GPU that loads the library holds it until the
- * process exits.  The call itself never calls cudaMalloc, cudaFree or any allocating routine.
+ * to its own pool, a plug-in whose host forbids allocations after start-up -- and therefore
+ * cannot hand the library a workspace.  The scratch the split-sequence decode kernel needs
+ * (partial outputs, their softmax statistics, arrival counters, the device copy of the lengths)
+ * lives in a fixed array of about 2.1 MB inside the library's device image; every GPU that loads
+ * the library holds it until the process exits.  The call itself never calls cudaMalloc, cudaFree
+ * or any allocating routine.  (Loading the library's device image is the CUDA runtime's business:
+ * with lazy module loading it happens at the first call on a device, and that is when the driver
+ * sets the array and the kernels up.  Make that first call at start-up, before the caller's own
+ * pool claims what is left of the device; every later call touches no allocator at all.)
  *
  * Computes, for each sequence b, full (retrieval) attention of one query token over the first
  * h_len[b] rows of the caller's stores:
@@ -257,8 +272,9 @@ int zz_profile_read(int kind, int64_t* launches, double* total_ms, int reset);
  * thread and stream, share the one array per device: it keeps the previous call's contents (the
  * call clears the counters it needs at zero itself), and two calls whose kernels may overlap on
  * the GPU race on it -- issue them on one stream, or order them yourself.  Asynchronous on
- * `stream`; h_len may be reused as soon as the call returns if it is pageable memory, and after
- * the stream reaches the copy if it is pinned. */
+ * `stream`: each call enqueues a copy of h_len and bakes the split plan it derives from h_len
+ * into the launch, so h_len may be reused as soon as the call returns if it is pageable memory,
+ * and after the stream reaches the copy if it is pinned. */
 int zz_decode_attn_static(const void* d_q, const void* d_k, const void* d_v, void* d_out,
                           const int32_t* h_len, int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
                           int32_t capacity, float softmax_scale, void* stream);

@@ -87,6 +87,7 @@ SYMBOLS = {
     "zz_cache_export": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, ctypes.POINTER(ctypes.c_int32), _vp]),
     "zz_cache_import": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp]),
     "zz_get_last_status": (_i32, [_vp, _vp]),
+    "zz_selftest_wait_timeout": (_i32, [_vp, _i32, _vp]),
     "zz_layer_mask_solve": (_i32, [_vp, _i32, _i32, _i32, ctypes.c_double, _vp, _vp, ctypes.POINTER(ctypes.c_double)]),
     "zz_decode_attn_static": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, ctypes.c_float, _vp]),
     "zz_decode_attn_static_limits": (_i32, [ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
@@ -172,14 +173,24 @@ def _stream_ptr(stream) -> Optional[int]:
     return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
 
 
+GUARD_BYTE = 0xA5
+
+
 class ZigzagCache:
-    """Owner of the device arena/workspace (torch allocations) and of the library handle."""
+    """Owner of the device arena/workspace (torch allocations) and of the library handle.
+
+    guard_bytes > 0 (a multiple of 256; `ZigzagCache.default_guard_bytes` when not given): the arena
+    and the workspace are each allocated with that many extra bytes on either side, filled with a
+    pattern; `guards_intact()` tells whether any kernel wrote outside the memory the library was
+    given, and `close()` raises if one did."""
+
+    default_guard_bytes = 0
 
     def __init__(self, n_layers: int, batch: int, n_q_heads: int, n_kv_heads: int, sink: int,
                  recent: int, layer_is_retrieval: Sequence[int], capacity: Sequence[int],
                  max_new_tokens: int, softmax_scale: Optional[float] = None,
                  kvhead_is_retrieval: Optional[np.ndarray] = None, head_dim: int = 128,
-                 device: str = "cuda:0", pool_pages: int = 0):
+                 device: str = "cuda:0", pool_pages: int = 0, guard_bytes: Optional[int] = None):
         import torch
         lib = load()
         self._lib = lib
@@ -208,9 +219,18 @@ class ZigzagCache:
             _check(lib.zz_cache_query(ctypes.byref(cfg), ctypes.byref(a), ctypes.byref(w)), "zz_cache_query")
         self.arena_bytes, self.workspace_bytes = int(a.value), int(w.value)
         self.device = torch.device(device)
+        g = int(self.default_guard_bytes if guard_bytes is None else guard_bytes)
+        assert g >= 0 and g % 256 == 0
+        self.guard_bytes = g
         with torch.cuda.device(self.device):
-            self._arena = torch.empty(self.arena_bytes, dtype=torch.uint8, device=self.device)
-            self._work = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=self.device)
+            self._arena_alloc = torch.empty(self.arena_bytes + 2 * g, dtype=torch.uint8, device=self.device)
+            self._work_alloc = torch.empty(self.workspace_bytes + 2 * g, dtype=torch.uint8, device=self.device)
+            if g:
+                for t in (self._arena_alloc, self._work_alloc):
+                    t[:g].fill_(GUARD_BYTE)
+                    t[t.numel() - g:].fill_(GUARD_BYTE)
+            self._arena = self._arena_alloc[g:g + self.arena_bytes]
+            self._work = self._work_alloc[g:g + self.workspace_bytes]
             h = ctypes.c_void_p(None)
             if self.pool_pages:
                 _check(lib.zz_cache_create_paged(ctypes.byref(cfg), self.pool_pages, self._arena.data_ptr(),
@@ -222,11 +242,26 @@ class ZigzagCache:
                        "zz_cache_create")
         self._h = h
 
+    def guards_intact(self) -> bool:
+        """True when no byte of the guard bands around arena and workspace has changed (synchronises)."""
+        import torch
+        g = self.guard_bytes
+        if not g:
+            return True
+        torch.cuda.synchronize(self.device)
+        for t in (self._arena_alloc, self._work_alloc):
+            if not bool((t[:g] == GUARD_BYTE).all()) or not bool((t[t.numel() - g:] == GUARD_BYTE).all()):
+                return False
+        return True
+
     # -- lifetime ---------------------------------------------------------------------------
     def close(self) -> None:
         if getattr(self, "_h", None):
+            intact = self.guards_intact() if self.guard_bytes else True
             self._lib.zz_cache_destroy(self._h)
             self._h = None
+            if not intact:
+                raise RuntimeError("a kernel wrote outside the arena or the workspace (guard band changed)")
 
     def __del__(self):
         try:
@@ -337,6 +372,11 @@ class ZigzagCache:
 
     def last_status(self, stream=None) -> int:
         return int(self._lib.zz_get_last_status(self._h, _stream_ptr(stream)))
+
+    def selftest_wait_timeout(self, max_polls: int = 1000, stream=None) -> None:
+        """One warp waits, bounded, on a barrier nothing completes; afterwards last_status() is ZZ_ERR_TIMEOUT."""
+        _check(self._lib.zz_selftest_wait_timeout(self._h, int(max_polls), _stream_ptr(stream)),
+               "zz_selftest_wait_timeout")
 
 
 def decode_attn_static(q, k, v, out, lens, softmax_scale: Optional[float] = None, stream=None) -> None:

@@ -54,7 +54,7 @@ using zz::SeqDesc;
 
 namespace {
 
-constexpr int kMaxSplits = 120;   // the decode kernel keeps per-split factors in 128-entry rows
+constexpr int kMaxSplits = zz::kDecodeMaxSplits;   // the decode kernel keeps per-split factors in 128-entry rows
 constexpr int kMaxSlots = 512;    // upper bound of CTAs a long-store decode plan may use (2 per SM)
 constexpr size_t kAlign = 256;
 
@@ -282,7 +282,12 @@ void plan_splits(const zz_cache* c, const int* n, int Hg, int* warps, int* chunk
     long long total = 0;
     for (int b = 0; b < c->B; ++b) total += n[b];
     split_start[0] = 0;
-    if (total * Hg <= (long long)c->num_sms * c->decode_short_tokens) {
+    // the short plan has one split per decode_short_tokens tokens: it serves a launch only if no
+    // sequence needs more splits than the kernel's merge can hold (one KV head and ~50K tokens would)
+    bool short_ok = c->decode_short_tokens > 0 && total * Hg <= (long long)c->num_sms * c->decode_short_tokens;
+    for (int b = 0; b < c->B && short_ok; ++b)
+        if ((n[b] + c->decode_short_tokens - 1) / c->decode_short_tokens > kMaxSplits) short_ok = false;
+    if (short_ok) {
         *warps = 8;
         for (int b = 0; b < c->B; ++b) {
             int s = (n[b] + c->decode_short_tokens - 1) / c->decode_short_tokens;
@@ -1234,6 +1239,19 @@ int zz_cache_import(zz_cache_t* c, int layer, int seq, int kind, const void* h_k
     if (e != cudaSuccess) return ZZ_ERR_CUDA;
     c->len[(size_t)layer * c->B + seq] = len;
     return ZZ_OK;
+}
+
+int zz_selftest_wait_timeout(zz_cache_t* c, int32_t max_polls, void* stream) {
+    if (!c || max_polls < 1 || max_polls > (1 << 16)) return ZZ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the flag sits in the spare bytes of the status section (word 0 status, word 16 append counter)
+    int* gave_up = c->d_status() + 32;
+    if (cudaMemsetAsync(gave_up, 0, sizeof(int), st) != cudaSuccess) return ZZ_ERR_CUDA;
+    if (zz::launch_wait_probe(c->d_status(), (unsigned int)max_polls, gave_up, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    int v = 0;
+    if (cudaMemcpyAsync(&v, gave_up, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ZZ_ERR_CUDA;
+    return v == 1 ? ZZ_OK : ZZ_ERR_CUDA;
 }
 
 int zz_get_last_status(zz_cache_t* c, void* stream) {

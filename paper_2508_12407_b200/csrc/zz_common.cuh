@@ -28,6 +28,13 @@ struct SeqDesc {
     int tbl;   // paged stores: first page-table entry of this (layer, sequence)
 };
 
+// Split limits of the decode kernel: the last CTA of a (sequence, head) merges the splits with the
+// per-split statistics held in rows of kDecodeSplitSlots floats of shared memory, the last slot of a
+// row being reserved for the reciprocal of the merged sum.  Host plans never exceed kDecodeMaxSplits.
+constexpr int kDecodeSplitSlots = 128;
+constexpr int kDecodeMaxSplits = 120;
+static_assert(kDecodeMaxSplits < kDecodeSplitSlots, "the merge keeps one spare slot per row");
+
 constexpr int kPageTokens = 128;
 constexpr long long kPageElems = 2LL * kPageTokens * kD;   // K block, then V block
 
@@ -67,7 +74,8 @@ struct DecodeParams {
     int kind;                // which group of the layer
     int ring;                // S+W
     int Hg, G, B;
-    int max_splits;
+    int max_splits;          // most splits any sequence of this launch has (<= kDecodeMaxSplits); the kernel
+                             // refuses a plan beyond it instead of overrunning its merge rows
     float scale_log2;        // softmax_scale * log2(e)
     // fused append (k_new != nullptr): the token at position len is taken from k_new/v_new
     // ([B][n_kv_total][128], model head order), written to its slot, and attended to
@@ -142,6 +150,8 @@ cudaError_t prefill_setup();
 // arena seen as rows of 128 bf16 (2-D); opaque 128-byte CUtensorMap objects
 cudaError_t launch_prefill(const PrefillParams& p, const void* tmap_q, const void* tmap_k,
                            const void* tmap_v, const void* tmap_arena, int n_items, cudaStream_t s);
+
+cudaError_t launch_wait_probe(int* status, unsigned int polls, int* gave_up, cudaStream_t s);
 
 void count_launch(int n = 1);
 

@@ -34,7 +34,7 @@ constexpr int kStageBytes = kBlk * kRowBytes;  // 4 KiB of K (and as much of V) 
 constexpr int kWarpSmem = kStages * 2 * kStageBytes;   // 24 KiB per warp
 // 4 warps: 96 KiB, two CTAs per SM (long contexts); 8 warps: 192 KiB, one CTA per SM (short
 // stores, where the per-warp chain of dependent steps is what costs)
-constexpr int kMaxSplitsSmem = 128;             // >= the host's split limit
+constexpr int kMaxSplitsSmem = kDecodeSplitSlots;   // merge rows; the host's split limit is below it
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return (uint32_t)__cvta_generic_to_shared(p);
@@ -167,6 +167,13 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     const int hg = local % p.Hg;
     const int split = local / p.Hg;
     const int nsplit = p.split_start[b + 1] - p.split_start[b];
+
+    // A plan with more splits than the merge rows hold is refused, not run: every CTA of the launch
+    // sees the same plan and returns before it touches a store, the scratch or the output.
+    if (nsplit > p.max_splits || p.max_splits > kDecodeMaxSplits) {
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, ZZ_ERR_UNSUPPORTED);
+        return;
+    }
 
     const bool fused = k_new_p != nullptr;
     const int len_old = len_p[b];

@@ -1,8 +1,8 @@
 // Decode attention for callers that must not allocate device memory.
 //
 // Some callers of this library run where cudaMalloc is off limits: inside a serving loop that
-// has handed every byte of the device to its own pool, in code that may be running under stream
-// capture, or in a plug-in whose host forbids driver allocations after start-up.  The regular
+// has handed every byte of the device to its own pool, or in a plug-in whose host forbids driver
+// allocations after start-up.  The regular
 // path asks such a caller for a workspace (zz_cache_query / zz_cache_create); this entry point
 // asks for nothing but the inputs and the output.  The split-sequence decode kernel still needs
 // scratch memory (per-split partial outputs, their softmax statistics, the arrival counters and

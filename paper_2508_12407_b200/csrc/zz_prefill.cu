@@ -62,6 +62,7 @@ struct Shared {
     uint64_t p_full[2];
     uint64_t o_full;
     uint32_t tmem_base;
+    uint32_t poll_limit;       // probes a wait may spend before it gives up (kMaxPolls in the product kernels)
     int abort_flag;
 };
 
@@ -92,7 +93,7 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
 // The first probe is inlined: a wait on a phase that has already completed costs one
 // try_wait, and only a real wait enters the polling loop.
 __device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, Shared* sh, int* status) {
-    const uint32_t limit = (*(volatile int*)&sh->abort_flag) ? kAbortPolls : kMaxPolls;
+    const uint32_t limit = (*(volatile int*)&sh->abort_flag) ? (uint32_t)kAbortPolls : (uint32_t)(*(volatile uint32_t*)&sh->poll_limit);
     for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try(bar, parity)) return true;
         if ((i & 4095u) == 4095u && (*(volatile int*)&sh->abort_flag)) break;
@@ -395,6 +396,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
             mbar_init(&sh.p_full[i], 128);
         }
         mbar_init(&sh.o_full, 1);
+        sh.poll_limit = kMaxPolls;
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -826,7 +828,31 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
     }
 }
 
+// Exercises the bounded wait on its failure path without any copy or MMA in flight: one warp waits
+// on a barrier of its own that nothing ever completes, the wait runs out after `polls` probes,
+// records ZZ_ERR_TIMEOUT in the status word and the kernel returns normally.
+__global__ void wait_probe_kernel(int* status, uint32_t polls, int* gave_up) {
+    __shared__ Shared sh;
+    if (threadIdx.x == 0) {
+        mbar_init(&sh.q_full, 1);
+        sh.poll_limit = polls;
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const bool ok = mbar_wait(&sh.q_full, 0, &sh, status);
+        *gave_up = ok ? 0 : 1;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_wait_probe(int* status, unsigned int polls, int* gave_up, cudaStream_t s) {
+    wait_probe_kernel<<<1, 32, 0, s>>>(status, polls, gave_up);
+    count_launch();
+    return cudaGetLastError();
+}
 
 static int g_num_sms = 0;
 

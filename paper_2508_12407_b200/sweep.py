@@ -89,35 +89,46 @@ def prefill_latency(arm: str, prompt: int, gen, reps: int = 3) -> float:
     return e0.elapsed_time(e1) * 1e3 / reps / prompt
 
 
+ARMS = ("original", "mixed", "exclusive")
+
+
+def run(lengths, decode_prompt: int = 16384, reps: int = 3, echo: bool = False):
+    """{"decode": {length: {arm: us/token}}, "prefill": {...}} for the given lengths."""
+    build.build()
+    binding.load()
+    gen = torch.Generator(device="cuda:0")
+    gen.manual_seed(inputs.BASE_SEED)
+    rows = {"decode": {}, "prefill": {}}
+    for n in lengths:
+        rows["decode"][n] = {a: decode_latency(a, decode_prompt, n, gen) for a in ARMS}
+        rows["prefill"][n] = {a: prefill_latency(a, n, gen, reps) for a in ARMS}
+        if echo:
+            print(json.dumps({"length": n, "decode_us_per_token": rows["decode"][n],
+                              "prefill_us_per_token": rows["prefill"][n]}), flush=True)
+    return rows
+
+
+def table(rows) -> str:
+    lines = ["| phase | length | original | mixed | exclusive | exclusive vs mixed | exclusive vs original |",
+             "|---|---:|---:|---:|---:|---:|---:|"]
+    for phase in ("decode", "prefill"):
+        for n, r in rows[phase].items():
+            lines.append(f"| {phase} | {n} | {r['original']:.1f} | {r['mixed']:.1f} | {r['exclusive']:.1f} | "
+                         f"{100 * (1 - r['exclusive'] / r['mixed']):.0f} % | {100 * (1 - r['exclusive'] / r['original']):.0f} % |")
+    return "\n".join(lines)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--out", default=None, help="write a markdown table here")
     ap.add_argument("--quick", action="store_true", help="lengths up to 4K only")
     args = ap.parse_args()
-    build.build()
-    binding.load()
-    gen = torch.Generator(device="cuda:0")
-    gen.manual_seed(inputs.BASE_SEED)
     lengths = [1024, 2048, 4096] if args.quick else [1024, 2048, 4096, 8192, 16384, 32768]
-    arms = ["original", "mixed", "exclusive"]
-    rows = {"decode": {}, "prefill": {}}
-    for n in lengths:
-        rows["decode"][n] = {a: decode_latency(a, 16384, n, gen) for a in arms}
-        rows["prefill"][n] = {a: prefill_latency(a, n, gen) for a in arms}
-        print(json.dumps({"length": n, "decode_us_per_token": rows["decode"][n],
-                          "prefill_us_per_token": rows["prefill"][n]}), flush=True)
-    lines = ["| phase | length | original | mixed | exclusive | exclusive vs mixed | exclusive vs original |",
-             "|---|---:|---:|---:|---:|---:|---:|"]
-    for phase in ("decode", "prefill"):
-        for n in lengths:
-            r = rows[phase][n]
-            lines.append(f"| {phase} | {n} | {r['original']:.1f} | {r['mixed']:.1f} | {r['exclusive']:.1f} | "
-                         f"{100 * (1 - r['exclusive'] / r['mixed']):.0f} % | {100 * (1 - r['exclusive'] / r['original']):.0f} % |")
-    table = "\n".join(lines)
-    print(table)
+    t = table(run(lengths, echo=True))
+    print(t)
     if args.out:
         with open(args.out, "w") as f:
-            f.write(table + "\n")
+            f.write(t + "\n")
 
 
 if __name__ == "__main__":

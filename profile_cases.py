@@ -1,6 +1,6 @@
 """Small, self-contained launches of each kernel for profiling under ncu.
 
-    python -m paper_2508_12407_b200.profile_cases --case decode_r [--n 32768] [--batch 1] [--reps 3]
+    python profile_cases.py --case decode_r [--n 32768] [--batch 1] [--reps 3]
 
 Each case holds well under a few GB on the device and its inputs exceed the 126 MB L2, so a
 capture of one to three launches ends by itself and its DRAM counters are meaningful.
@@ -11,11 +11,15 @@ layers alternate retrieval / streaming, one grid per kind, as the benchmark laun
 from __future__ import annotations
 
 import argparse
+import os
+import sys
 
 import numpy as np
 import torch
 
-from . import binding, build
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+
+from paper_2508_12407_b200 import binding, build  # noqa: E402
 
 
 def main():

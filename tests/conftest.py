@@ -24,3 +24,31 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _guard_bands(request):
+    """GPU tests give every cache 64 KiB of patterned guard band on either side of its arena and of
+    its workspace (a stand-in for a memory checker): `close()` raises when a kernel wrote there, and
+    caches a test leaves open are checked when the test ends."""
+    if "gpu" not in request.keywords:
+        yield
+        return
+    from paper_2508_12407_b200 import binding
+    live = []
+    orig_init = binding.ZigzagCache.__init__
+
+    def tracking_init(self, *a, **kw):
+        orig_init(self, *a, **kw)
+        live.append(self)
+
+    binding.ZigzagCache.default_guard_bytes = 64 * 1024
+    binding.ZigzagCache.__init__ = tracking_init
+    try:
+        yield
+    finally:
+        binding.ZigzagCache.__init__ = orig_init
+        binding.ZigzagCache.default_guard_bytes = 0
+    for c in live:
+        if getattr(c, "_h", None):
+            assert c.guards_intact(), "a kernel wrote outside the arena or the workspace"

@@ -27,11 +27,13 @@ def layer_kv_kinds(kinds, Hkv, kvk, l):
 
 
 def run_append_decode(L, B, Hq, Hkv, S, W, kinds, lens, n_decode, seed, kvk=None, chunk_cap=300,
-                      check_every=1, pool_pages=0):
+                      check_every=1, pool_pages=0, tune=None):
     D = 128
     scale = 1.0 / np.sqrt(D)
     cap = [int(n) + n_decode for n in lens]
-    cache = make(L, B, Hq, Hkv, S, W, kinds, cap, kvk, pool_pages=pool_pages)
+    cache = make(L, B, Hq, Hkv, S, W, kinds, cap, kvk, max_new=max(4096, chunk_cap * B), pool_pages=pool_pages)
+    for key, value in (tune or {}).items():
+        cache.tune(key, value)
     w = inputs.Workload("t", L, B, Hq, Hkv, D, S, W, int(sum(kinds)), 0, 0, n_decode, seed=seed)
     orc = [[OracleSeq(Hkv, D, S, W, cap[b], layer_kv_kinds(kinds, Hkv, kvk, l)) for b in range(B)]
            for l in range(L)]
@@ -104,6 +106,36 @@ def test_group_sizes(Hq, Hkv):
 def test_many_splits_long_context():
     # long enough that the retrieval layer is split over many CTAs and merged
     run_append_decode(2, 1, 8, 2, 128, 256, [1, 0], [9000], 3, seed=5, chunk_cap=4000)
+
+
+# One KV head in the group and a store of about 50K tokens: at 384 tokens per split the short plan
+# would need more splits (129-148) than the kernel's merge rows hold, so the planner must switch to
+# the long plan there, and the short plan with a split count just below the limit must be right too.
+@pytest.mark.parametrize("n", [40000, 46000, 50000, 56832 - 2])
+def test_one_kv_head_store_near_the_split_limit(n):
+    run_append_decode(2, 1, 4, 1, 128, 256, [1, 0], [n], 2, seed=n, chunk_cap=8192)
+
+
+def test_one_kv_head_ring_near_the_split_limit():
+    # the same plan question on a streaming layer whose ring is that large
+    run_append_decode(2, 1, 4, 1, 128, 52000, [0, 1], [53000], 2, seed=53, chunk_cap=8192)
+
+
+@pytest.mark.parametrize("n", [50000, 56000])
+def test_mixed_layer_with_one_retrieval_head_near_the_split_limit(n):
+    kvk = np.array([[1, 0], [0, 1]], dtype=np.uint8)
+    run_append_decode(2, 1, 8, 2, 128, 256, [0, 0], [n], 2, seed=n + 1, kvk=kvk, chunk_cap=8192)
+
+
+def test_one_long_one_short_sequence_near_the_split_limit():
+    run_append_decode(1, 2, 4, 1, 128, 256, [1], [52000, 300], 2, seed=523, chunk_cap=8192)
+
+
+@pytest.mark.parametrize("short,n", [(512, 70000), (1024, 100000), (1024, 130000)])
+def test_short_plan_threshold_tuned_up(short, n):
+    # 137 splits of 512 tokens would overrun the merge rows (long plan instead); 98 splits of 1024
+    # tokens is a legal short plan with many splits; 127 of 1024 is again past the limit
+    run_append_decode(1, 1, 4, 1, 128, 256, [1], [n], 2, seed=n, chunk_cap=8192, tune={"decode_short_tokens": short})
 
 
 def test_ragged_batch():
