@@ -40,7 +40,10 @@ constexpr int kThreads = 384;                // three warpgroups: softmax tile 0
 constexpr int kWarpTma = 8, kWarpMma = 9;
 constexpr int kRegsSoftmax = 200, kRegsAux = 104;  // 200 * 256 + 104 * 128 = 64512 registers, what the launch allocates (168 * 384)
 constexpr int kEpiBytes = 8 * 4096;          // output staging: 16 rows of 256 B per softmax warp
-constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + kEpiBytes + 1024;
+constexpr int kMaxOrder = 768;               // items of one CTA that can be re-ordered (2 bytes each)
+constexpr int kMaxOrderKeys = 1024;          // distinct (sequence, KV head) keys the re-ordering handles
+constexpr int kOrderBytes = kMaxOrder * 2;
+constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + kEpiBytes + kOrderBytes + 1024;
 constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr uint32_t kAbortPolls = 1u << 10;
 constexpr float kRescaleThreshold = 8.f;    // log2 units of slack before O is rescaled
@@ -363,6 +366,15 @@ __device__ __forceinline__ Item get_item(const PrefillParams& p, int idx) {
     it.n_tiles = it.plan.n_total;
     return it;
 }
+// (sequence, KV head) of an item as one number: items with equal keys read the same K/V rows
+__device__ __forceinline__ int item_key(const PrefillParams& p, int idx) {
+    const int pairs = (p.G + 1) >> 1;
+    const int per_tile = p.Hg * pairs;
+    const int gt = p.total_tiles - 1 - idx / per_tile;
+    int b = 0;
+    while (b + 1 < p.B && gt >= p.tile_start[b + 1]) ++b;
+    return b * p.Hg + (idx % per_tile) / pairs;
+}
 
 // kPersistent = false: one item per CTA (grid = items, for launches with no more items than SMs);
 // the item loops below then run once and every running counter folds to a constant.  Persistent
@@ -383,6 +395,68 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
 
     const int n_items = p.n_items;
     const uint32_t sm_epi = smem_base + 2 * kTileBytes + kStages * kTileBytes;   // output staging
+
+    // ---- this CTA's items and the order it takes them in ------------------------------------------
+    // The static schedule hands CTA c the items k * grid + snake(c), k = 0 .. n_mine - 1, of the
+    // long-first numbering (equal work per CTA).  A retrieval launch walks its share sorted by
+    // (sequence, KV head) instead: all CTAs then stream the same one or two KV heads at any time, whose
+    // K/V rows fit the L2, instead of all heads at once (K/V came from HBM 4-11 times over).  The sort
+    // is stable, so within a head the long items still come first.
+    int n_mine = 1;
+    bool use_order = false;
+    if (kPersistent) {
+        const int g = (int)gridDim.x, full = n_items / g, rem = n_items % g;
+        const int pos = (full & 1) ? g - 1 - (int)blockIdx.x : (int)blockIdx.x;
+        n_mine = full + (pos < rem ? 1 : 0);
+        use_order = p.kind == ZZ_KIND_RETRIEVAL && n_mine > 2 && n_mine <= kMaxOrder && p.B * p.Hg <= kMaxOrderKeys &&
+                    p.B * p.Hg > 1;
+    }
+    unsigned char* const smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    uint16_t* const sm_order = reinterpret_cast<uint16_t*>(smem_gen + 2 * kTileBytes + kStages * kTileBytes + kEpiBytes);
+    if (kPersistent && use_order && warp == 10) {
+        uint16_t* const cnt = reinterpret_cast<uint16_t*>(smem_gen + 2 * kTileBytes + kStages * kTileBytes);  // scratch: the staging area
+        const int nkeys = p.B * p.Hg;
+        for (int i = lane; i < nkeys; i += 32) cnt[i] = 0;
+        __syncwarp();
+        for (int k0 = 0; k0 < n_mine; k0 += 32) {          // how many of my items each key has
+            const int k = k0 + lane;
+            const bool valid = k < n_mine;
+            const int key = valid ? item_key(p, item_index(k, n_items)) : -1 - lane;
+            const unsigned m = __match_any_sync(0xffffffffu, key);
+            if (valid && lane == __ffs(m) - 1) cnt[key] += (uint16_t)__popc(m);
+            __syncwarp();
+        }
+        int carry = 0;
+        for (int i0 = 0; i0 < nkeys; i0 += 32) {             // exclusive prefix sum: first position of each key
+            const int i = i0 + lane;
+            const int v = i < nkeys ? cnt[i] : 0;
+            int incl = v;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            if (i < nkeys) cnt[i] = (uint16_t)(carry + incl - v);
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+            __syncwarp();
+        }
+        for (int k0 = 0; k0 < n_mine; k0 += 32) {          // stable scatter
+            const int k = k0 + lane;
+            const bool valid = k < n_mine;
+            const int key = valid ? item_key(p, item_index(k, n_items)) : -1 - lane;
+            const unsigned m = __match_any_sync(0xffffffffu, key);
+            if (valid) sm_order[cnt[key] + __popc(m & ((1u << lane) - 1u))] = (uint16_t)k;
+            __syncwarp();
+            if (valid && lane == __ffs(m) - 1) cnt[key] += (uint16_t)__popc(m);
+            __syncwarp();
+        }
+    }
+    // item k of this CTA (or -1 past the last one)
+    auto my_item = [&](int k) -> int {
+        if (!kPersistent) return (int)blockIdx.x;
+        if (k >= n_mine) return -1;
+        return item_index(use_order ? (int)sm_order[k] : k, n_items);
+    };
 
     if (threadIdx.x == 0) {
         mbar_init(&sh.q_full, 1);
@@ -420,7 +494,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
             uint32_t u_glob = 0;                      // K/V pairs loaded so far (all items)
             for (int k = 0;; ++k) {
                 if (!kPersistent && k > 0) break;
-                const int idx = kPersistent ? item_index(k, n_items) : (int)blockIdx.x;
+                const int idx = my_item(k);
                 if (idx < 0) break;
                 const Item it = get_item(p, idx);
                 const SeqDesc sd = p.desc[it.b];
@@ -491,7 +565,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
             uint32_t ph[2] = {0, 0};      // S/P tiles handled per query tile (tile 1 only in items that have it)
             for (int k = 0;; ++k) {
                 if (!kPersistent && k > 0) break;
-                const int idx = kPersistent ? item_index(k, n_items) : (int)blockIdx.x;
+                const int idx = my_item(k);
                 if (idx < 0) break;
                 const Item it = get_item(p, idx);
                 const int n_tiles = __shfl_sync(0xffffffffu, it.n_tiles, 0);
@@ -570,7 +644,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
         uint32_t ph = 0;                                // S/P tiles of this query tile handled so far
         for (int k = 0;; ++k) {
             if (!kPersistent && k > 0) break;
-            const int item_idx = kPersistent ? item_index(k, n_items) : (int)blockIdx.x;
+            const int item_idx = my_item(k);
             if (item_idx < 0) break;
             const Item it = get_item(p, item_idx);
             if (t == 1 && !it.active1) continue;
