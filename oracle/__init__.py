@@ -57,6 +57,14 @@ def _load() -> ctypes.CDLL:
     lib.zzo_layer_mask_enumerate.restype = i32
     lib.zzo_quantile_split.argtypes = [vp, i32, i32, vp]
     lib.zzo_quantile_split.restype = i32
+    lib.zzo_e4m3_value.argtypes = [ctypes.c_uint8]
+    lib.zzo_e4m3_value.restype = dbl
+    lib.zzo_e4m3_encode.argtypes = [dbl]
+    lib.zzo_e4m3_encode.restype = ctypes.c_uint8
+    lib.zzo_fp8_quantize_rows.argtypes = [vp, i64, i32, vp, vp]
+    lib.zzo_fp8_quantize_rows.restype = i32
+    lib.zzo_fp8_dequantize_rows.argtypes = [vp, vp, i64, i32, vp]
+    lib.zzo_fp8_dequantize_rows.restype = i32
     _lib = lib
     return lib
 
@@ -155,6 +163,75 @@ def layer_mask_enumerate(alpha: np.ndarray, head_is_retr: np.ndarray, p: int, om
     if rc != 0:
         raise ValueError(f"zzo_layer_mask_enumerate failed: {rc}")
     return out, float(best.value), float(second.value)
+
+
+def e4m3_value(code: int) -> float:
+    return float(_load().zzo_e4m3_value(int(code) & 0xFF))
+
+
+def e4m3_encode(y: float) -> int:
+    return int(_load().zzo_e4m3_encode(float(y)))
+
+
+def fp8_quantize_rows(x: np.ndarray):
+    """bf16 bit patterns [..., D] -> (E4M3 codes uint8 [..., D], scale bytes uint8 [...])."""
+    x = _u16(x)
+    D = x.shape[-1]
+    n = x.size // D
+    codes = np.empty(x.shape, dtype=np.uint8)
+    scale = np.empty(x.shape[:-1], dtype=np.uint8)
+    rc = _load().zzo_fp8_quantize_rows(_ptr(x), n, D, _ptr(codes), _ptr(scale))
+    if rc != 0:
+        raise ValueError(f"zzo_fp8_quantize_rows failed: {rc}")
+    return codes, scale
+
+
+def fp8_dequantize_rows(codes: np.ndarray, scale: np.ndarray) -> np.ndarray:
+    """Stored values as float64: value(code) * 2^(scale - 127)."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    scale = np.ascontiguousarray(scale, dtype=np.uint8)
+    D = codes.shape[-1]
+    assert codes.shape[:-1] == scale.shape
+    out = np.empty(codes.shape, dtype=np.float64)
+    rc = _load().zzo_fp8_dequantize_rows(_ptr(codes), _ptr(scale), codes.size // D, D, _ptr(out))
+    if rc != 0:
+        raise ValueError(f"zzo_fp8_dequantize_rows failed: {rc}")
+    return out
+
+
+def fp8_stored_as_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """What rows read back as after FP8 storage, as bf16 bit patterns.  The stored values have four
+    significant bits and a power-of-two scale, so they are bf16 numbers exactly (checked)."""
+    codes, scale = fp8_quantize_rows(x)
+    v = fp8_dequantize_rows(codes, scale)
+    f = v.astype(np.float32)
+    bits = (f.view(np.uint32) >> np.uint32(16)).astype(np.uint16)
+    back = (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    if not np.array_equal(back, v):
+        raise ValueError("a stored FP8 value is not a bf16 number (exponent out of range)")
+    return bits
+
+
+class Fp8Store:
+    """Retrieval KV store in FP8: slot j holds the codes and the scale byte of token j."""
+
+    def __init__(self, Hkv: int, D: int, cap: int):
+        self.Hkv, self.D, self.cap = Hkv, D, cap
+        self.k = np.zeros((Hkv, cap, D), dtype=np.uint8)
+        self.v = np.zeros((Hkv, cap, D), dtype=np.uint8)
+        self.k_scale = np.zeros((Hkv, cap), dtype=np.uint8)
+        self.v_scale = np.zeros((Hkv, cap), dtype=np.uint8)
+        self.len = 0
+
+    def append(self, k_new: np.ndarray, v_new: np.ndarray) -> None:
+        C = k_new.shape[0]
+        if self.len + C > self.cap:
+            raise ValueError("retrieval store overflow")
+        for src, codes, scales in ((k_new, self.k, self.k_scale), (v_new, self.v, self.v_scale)):
+            c, s = fp8_quantize_rows(np.ascontiguousarray(_u16(src).transpose(1, 0, 2)))
+            codes[:, self.len:self.len + C] = c
+            scales[:, self.len:self.len + C] = s
+        self.len += C
 
 
 class RingStore:

@@ -306,3 +306,88 @@ int zzo_quantile_split(const double* alpha, int n, int n_streaming, uint8_t* is_
     }
     return ZZO_OK;
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * FP8 storage of retrieval KV rows (the paper has no such variant; this is the reading the
+ * library documents, written out as its definition).
+ *
+ * A row is the 128 (in general D) bf16 values of one token and one KV head.  It is stored as
+ * D codes in the OCP 8-bit floating-point format E4M3 (1 sign, 4 exponent bits of bias 7, 3
+ * mantissa bits; no infinities; largest finite magnitude 448 = 1.75 * 2^8; S.1111.111 is NaN)
+ * and one scale byte e (an exponent-only number, value 2^(e - 127)):
+ *     amax = max_d |x_d|;  write amax = m * 2^k with 1 <= m < 2 (k taken from the exponent field
+ *     of the bf16 bits; a zero or subnormal amax counts as k = -127);
+ *     e = clamp(k + 127 - 8 + (m > 1.75 ? 1 : 0), 1, 254): the smallest power of two with
+ *     amax / 2^(e-127) <= 448, so nothing saturates;
+ *     code_d = E4M3 nearest to x_d / 2^(e-127), ties to the even code, magnitudes beyond 448
+ *     (only possible through the clamp) to 448.
+ * The stored value of the element is value(code_d) * 2^(e-127), exactly.
+ * --------------------------------------------------------------------------------------------- */
+
+/* value of one E4M3 code (NaN codes are never produced; they decode to 0 here) */
+double zzo_e4m3_value(uint8_t c) {
+    const int s = c >> 7, e = (c >> 3) & 15, m = c & 7;
+    double v;
+    if (e == 15 && m == 7) return 0.0;
+    if (e == 0) v = ldexp((double)m / 8.0, -6);
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return s ? -v : v;
+}
+
+/* nearest E4M3 code of y, ties to even, saturating at +-448 */
+uint8_t zzo_e4m3_encode(double y) {
+    const uint8_t sign = (y < 0.0 || (y == 0.0 && signbit(y))) ? 0x80 : 0x00;
+    double a = fabs(y);
+    if (!(a == a)) return (uint8_t)(sign | 0x7E);
+    if (a >= 448.0) return (uint8_t)(sign | 0x7E);
+    if (a == 0.0) return sign;
+    int ex;
+    (void)frexp(a, &ex);                /* a = f * 2^ex, 0.5 <= f < 1  ->  floor(log2 a) = ex - 1 */
+    int e = ex - 1;
+    if (e < -6) e = -6;                 /* subnormal range shares the quantum of the smallest normal */
+    const double quantum = ldexp(1.0, e - 3);
+    double n = nearbyint(a / quantum);  /* default rounding mode: to nearest, ties to even */
+    if (n >= 16.0) { n = 8.0; e += 1; }
+    int biased, mant;
+    if (n >= 8.0) { biased = e + 7; mant = (int)n - 8; }
+    else { biased = 0; mant = (int)n; } /* only reachable with e == -6 */
+    if (biased > 15 || (biased == 15 && mant == 7)) return (uint8_t)(sign | 0x7E);
+    return (uint8_t)(sign | (biased << 3) | mant);
+}
+
+/* scale byte of a row of D bf16 values */
+uint8_t zzo_fp8_scale_byte(const uint16_t* row, int D) {
+    unsigned amax = 0;
+    for (int d = 0; d < D; ++d) {
+        const unsigned a = row[d] & 0x7FFFu;
+        if (a > amax) amax = a;
+    }
+    const int k_biased = (int)(amax >> 7);          /* exponent field: k + 127 (0 for zero / subnormal) */
+    const int mant = (int)(amax & 0x7F);            /* m = 1 + mant / 128; 1.75 <-> 0x60 */
+    int e = k_biased - 8 + (mant > 0x60 ? 1 : 0);
+    if (e < 1) e = 1;
+    if (e > 254) e = 254;
+    return (uint8_t)e;
+}
+
+/* rows [n][D] bf16 bits -> codes [n][D], scale bytes [n] */
+int zzo_fp8_quantize_rows(const uint16_t* x, int64_t n, int D, uint8_t* codes, uint8_t* scale) {
+    if (!x || !codes || !scale || n < 0 || D <= 0) return ZZO_BAD_ARG;
+    for (int64_t r = 0; r < n; ++r) {
+        const uint16_t* row = x + (size_t)r * D;
+        const uint8_t e = zzo_fp8_scale_byte(row, D);
+        scale[r] = e;
+        for (int d = 0; d < D; ++d)
+            codes[(size_t)r * D + d] = zzo_e4m3_encode(ldexp(bf16_to_f64(row[d]), 127 - (int)e));
+    }
+    return ZZO_OK;
+}
+
+/* stored values as fp64: out[r][d] = value(code) * 2^(scale - 127) */
+int zzo_fp8_dequantize_rows(const uint8_t* codes, const uint8_t* scale, int64_t n, int D, double* out) {
+    if (!codes || !scale || !out || n < 0 || D <= 0) return ZZO_BAD_ARG;
+    for (int64_t r = 0; r < n; ++r)
+        for (int d = 0; d < D; ++d)
+            out[(size_t)r * D + d] = ldexp(zzo_e4m3_value(codes[(size_t)r * D + d]), (int)scale[r] - 127);
+    return ZZO_OK;
+}

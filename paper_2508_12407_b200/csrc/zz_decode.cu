@@ -473,7 +473,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     // per-split factors through shared memory while those loads are in flight.
     float* sm_m = reinterpret_cast<float*>(smem);            // [16][128] running max per split
     float* sm_f = sm_m + 16 * kMaxSplitsSmem;                // [16][128] sum, then factor
-    constexpr int kRound = 32;                               // splits whose partials are held at once
+    constexpr int kRound = 40;                               // splits whose partials are held at once (one round for the usual 37 of a 32K store)
     for (int row0 = 0; row0 < G; row0 += kWarps) {
         const int row = row0 + warp;                         // this warp's row (4 dims per lane)
         const bool row_ok = row < G;
