@@ -207,7 +207,8 @@ class Arm:
             heads_R = int(self.kvk.sum()) if self.kvk is not None else int(np.sum(self.kinds)) * Hkv
             pool_pages = heads_R * sum((c + 127) // 128 for c in cap)
         self.cache = binding.ZigzagCache(L, B, Hq, Hkv, w.sink, w.recent, self.kinds, cap, max(B, B * self.C),
-                                         kvhead_is_retrieval=self.kvk, device=str(dev), pool_pages=pool_pages)
+                                         kvhead_is_retrieval=self.kvk, device=str(dev), pool_pages=pool_pages,
+                                         kv_fp8=args.kv == "fp8")
         if args.decode_overlap >= 0:
             self.cache.tune("decode_overlap", args.decode_overlap)
         if share_from is not None:
@@ -336,7 +337,9 @@ class Arm:
         # decode bytes per step: K and V of the visible tokens + q + o + the appended rows (read + write).
         # The rings' share is algorithmic traffic too, but the kernel keeps it in the L2 on purpose
         # (evict-last), so it is also reported apart from what must come from HBM.
-        bytes_R = fr * float((2 * Hkv * avg_n * D * 2).sum())
+        # a retrieval row is 128 bf16 values, or 128 FP8 codes and a scale byte
+        row_bytes = (D + 1) if self.args.kv == "fp8" else D * 2
+        bytes_R = fr * float((2 * Hkv * avg_n * row_bytes).sum())
         bytes_S = fs * float((2 * Hkv * np.minimum(avg_n, ring) * D * 2).sum())
         bytes_io = L * B * (2 * Hq * D * 2 + 4 * Hkv * D * 2)
         return {"flops_R": flops_R, "flops_S": flops_S, "fr": fr, "fs": fs, "base_len": base_len,
@@ -387,7 +390,7 @@ def rooflines(arm, r, K, p, traffic):
     prof, steps_dec, n_chunks = r["prof"], arm.steps_dec, arm.n_chunks
     nR_layers = int(arm.kinds.sum()) if arm.kvk is None else None
     overlap3 = arm.args.decode_overlap in (-1, 3)
-    tkey = w.name + ("+mixed" if arm.mixed else "") + ("+paged" if arm.args.paged else "")
+    tkey = w.name + ("+mixed" if arm.mixed else "") + ("+paged" if arm.args.paged else "") + ("+fp8" if arm.args.kv == "fp8" else "")
 
     def roof(kind_name, bound, achieved, peak, unit, traffic_key):
         t = traffic.get(f"{tkey}.{traffic_key}") if overlap3 else None
@@ -404,7 +407,8 @@ def rooflines(arm, r, K, p, traffic):
         else:
             avg_n = wk["base_len"] + ((arm.warm_rounds + (K + 1) / 2.0) * steps_dec)
         heads_R = Hkv if arm.kvk is None else (w.mixed_retrieval_kv_heads or Hkv // 2)
-        bytes_launch = float((2 * heads_R * avg_n * D * 2).sum()) + B * heads_R * (Hq // Hkv) * D * 2 * 2
+        row_bytes = (D + 1) if arm.args.kv == "fp8" else D * 2
+        bytes_launch = float((2 * heads_R * avg_n * row_bytes).sum()) + B * heads_R * (Hq // Hkv) * D * 2 * 2
         # with the default launch mode one grid covers all retrieval layers of a step
         # (mixed arm: one grid covers the retrieval heads of every layer)
         layers_per_launch = (nR_layers if arm.kvk is None else L) if overlap3 else 1
@@ -484,7 +488,8 @@ def summary(arm, r, K, world, p, traffic):
 def config_of(arm, world):
     w = arm.w
     a = arm.args
-    return {"workload": w.name + ("+mixed" if arm.mixed else "") + ("+paged" if a.paged else "") + (f"+graph{a.graph}" if a.graph else ""),
+    return {"workload": w.name + ("+mixed" if arm.mixed else "") + ("+paged" if a.paged else "") + ("+fp8kv" if a.kv == "fp8" else "") + (f"+graph{a.graph}" if a.graph else ""),
+            "retrieval_kv": "fp8 e4m3 codes + one power-of-two scale byte per token and head" if a.kv == "fp8" else "bf16",
             "layers": w.n_layers, "batch": w.batch, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
             "sink": w.sink, "recent": w.recent, "retrieval_layers": int(arm.kinds.sum()) if arm.kvk is None else None,
             "retrieval_kv_heads_per_layer": None if arm.kvk is None else int(arm.kvk.sum() // w.n_layers),
@@ -698,6 +703,8 @@ def main():
     ap.add_argument("--workload", default="cfg5", choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--paged", action="store_true",
                     help="retrieval stores in 128-token pages from a shared pool (a variant, not the default)")
+    ap.add_argument("--kv", default="bf16", choices=["bf16", "fp8"],
+                    help="storage of the retrieval stores (fp8: E4M3 codes + a scale byte per token and head; a variant)")
     ap.add_argument("--graph", type=int, default=0, metavar="N",
                     help="replay the decode step from a CUDA graph, re-captured every N steps (0: plain launches)")
     ap.add_argument("--decode-steps", type=int, default=-1, help="override the workload's decode steps")

@@ -80,6 +80,8 @@ typedef struct zz_config {
                                            (overrides the layer mask; a layer holding both
                                            kinds runs the two-pass mixed-head path)             */
     const int32_t* capacity;            /* [batch] max tokens per sequence in retrieval stores  */
+    int32_t retrieval_kv_fp8;           /* 0: retrieval stores hold the bf16 rows as given; 1: they
+                                           hold FP8 rows (see "FP8 retrieval stores" below)        */
 } zz_config_t;
 
 /* Library version (major*10000 + minor*100 + patch). */
@@ -203,6 +205,29 @@ int zz_decode_step_all_host(zz_cache_t* cache, const void* h_q, const void* h_k,
 int zz_prefill_host(zz_cache_t* cache, int layer, const void* h_q, const void* h_k,
                     const void* h_v, void* h_out, const int32_t* h_n_new, void* d_stage,
                     size_t stage_bytes, void* stream);
+
+/* FP8 retrieval stores (cfg.retrieval_kv_fp8 = 1; a variant the paper does not describe -- its
+ * motivation, the size of the KV cache, is the Introduction's second paragraph).  Every row that
+ * enters a retrieval store (one token, one KV head, K or V) is stored as 128 codes in the 8-bit
+ * floating-point format E4M3 (1 sign, 4 exponent bits of bias 7, 3 mantissa bits, largest magnitude
+ * 448, no infinities) plus one scale byte e that stands for 2^(e - 127):
+ *   amax = the row's largest magnitude = m * 2^k, 1 <= m < 2;  e = k + 127 - 8 (+ 1 if m > 1.75),
+ *   at least 1: the smallest power of two that brings amax to at most 448, so nothing saturates;
+ *   code = the E4M3 number nearest to x / 2^(e-127), ties to the even code.
+ * The stored value is code * 2^(e-127), exactly, and attention over the store uses those values:
+ * 258 bytes per token and head instead of 512.  Queries, probabilities and accumulation are as
+ * with bf16 stores.  What attends to what: a decode step stores its token first, so the query
+ * sees its own token as stored; a prefill chunk sees earlier tokens as stored and its own tokens
+ * as given (bf16), and is stored afterwards by zz_kv_append.  Streaming rings stay bf16.  Not
+ * available together with paged stores (ZZ_ERR_UNSUPPORTED).  zz_cache_export / zz_cache_import
+ * refuse the retrieval group of such a cache (ZZ_ERR_UNSUPPORTED); the two calls below move its
+ * bytes: h_k_codes/h_v_codes [n_retrieval_heads, capacity[seq], 128] uint8 and h_k_scale/h_v_scale
+ * [n_retrieval_heads, capacity[seq]] uint8, heads in ascending KV-head order, slot j = token j.
+ * Both synchronise the stream. */
+int zz_cache_export_fp8(zz_cache_t* cache, int layer, int seq, void* h_k_codes, void* h_v_codes,
+                        void* h_k_scale, void* h_v_scale, int32_t* h_len, void* stream);
+int zz_cache_import_fp8(zz_cache_t* cache, int layer, int seq, const void* h_k_codes, const void* h_v_codes,
+                        const void* h_k_scale, const void* h_v_scale, int32_t len, void* stream);
 
 /* Snapshot of one store, for tests and checkpointing.  `kind` selects the KV-head group
  * of the layer (ZZ_KIND_RETRIEVAL / ZZ_KIND_STREAMING; an exclusive layer has only one).

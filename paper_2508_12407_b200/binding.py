@@ -42,6 +42,7 @@ class ZZConfig(ctypes.Structure):
         ("layer_is_retrieval", ctypes.c_void_p),
         ("kvhead_is_retrieval", ctypes.c_void_p),
         ("capacity", ctypes.c_void_p),
+        ("retrieval_kv_fp8", ctypes.c_int32),
     ]
 
 
@@ -86,6 +87,8 @@ SYMBOLS = {
                                      ctypes.POINTER(ctypes.c_int32)]),
     "zz_cache_export": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, ctypes.POINTER(ctypes.c_int32), _vp]),
     "zz_cache_import": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp]),
+    "zz_cache_export_fp8": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp, _vp, ctypes.POINTER(ctypes.c_int32), _vp]),
+    "zz_cache_import_fp8": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _vp]),
     "zz_get_last_status": (_i32, [_vp, _vp]),
     "zz_selftest_wait_timeout": (_i32, [_vp, _i32, _vp]),
     "zz_layer_mask_solve": (_i32, [_vp, _i32, _i32, _i32, ctypes.c_double, _vp, _vp, ctypes.POINTER(ctypes.c_double)]),
@@ -190,7 +193,8 @@ class ZigzagCache:
                  recent: int, layer_is_retrieval: Sequence[int], capacity: Sequence[int],
                  max_new_tokens: int, softmax_scale: Optional[float] = None,
                  kvhead_is_retrieval: Optional[np.ndarray] = None, head_dim: int = 128,
-                 device: str = "cuda:0", pool_pages: int = 0, guard_bytes: Optional[int] = None):
+                 device: str = "cuda:0", pool_pages: int = 0, guard_bytes: Optional[int] = None,
+                 kv_fp8: bool = False):
         import torch
         lib = load()
         self._lib = lib
@@ -208,7 +212,8 @@ class ZigzagCache:
         cfg = ZZConfig(n_layers, batch, n_q_heads, n_kv_heads, head_dim, sink, recent,
                        int(max_new_tokens), scale,
                        self._kinds.ctypes.data, None if self._kvk is None else self._kvk.ctypes.data,
-                       self._cap.ctypes.data)
+                       self._cap.ctypes.data, 1 if kv_fp8 else 0)
+        self.kv_fp8 = bool(kv_fp8)
         self._cfg = cfg
         a, w = ctypes.c_size_t(0), ctypes.c_size_t(0)
         self.pool_pages = int(pool_pages)
@@ -359,6 +364,26 @@ class ZigzagCache:
         _check(self._lib.zz_cache_export(self._h, layer, seq, kind, _np_ptr(k), _np_ptr(v), _np_ptr(pos),
                                          ctypes.byref(ln), _stream_ptr(stream)), "zz_cache_export")
         return k, v, pos, int(ln.value)
+
+    def export_fp8(self, layer: int, seq: int, stream=None):
+        """FP8 retrieval group: (k codes, v codes uint8 [heads, cap, 128], k scale, v scale uint8 [heads, cap], len)."""
+        nh, ns = self.export_shape(layer, seq, KIND_RETRIEVAL)
+        k = np.zeros((nh, ns, self.head_dim), dtype=np.uint8)
+        v = np.zeros_like(k)
+        ks = np.zeros((nh, ns), dtype=np.uint8)
+        vs = np.zeros_like(ks)
+        ln = ctypes.c_int32(0)
+        _check(self._lib.zz_cache_export_fp8(self._h, layer, seq, _np_ptr(k), _np_ptr(v), _np_ptr(ks), _np_ptr(vs),
+                                             ctypes.byref(ln), _stream_ptr(stream)), "zz_cache_export_fp8")
+        return k, v, ks, vs, int(ln.value)
+
+    def import_fp8(self, layer: int, seq: int, k, v, ks, vs, length: int, stream=None) -> None:
+        nh, ns = self.export_shape(layer, seq, KIND_RETRIEVAL)
+        k, v = np.ascontiguousarray(k, dtype=np.uint8), np.ascontiguousarray(v, dtype=np.uint8)
+        ks, vs = np.ascontiguousarray(ks, dtype=np.uint8), np.ascontiguousarray(vs, dtype=np.uint8)
+        assert k.shape == (nh, ns, self.head_dim) and v.shape == k.shape and ks.shape == (nh, ns) and vs.shape == ks.shape
+        _check(self._lib.zz_cache_import_fp8(self._h, layer, seq, _np_ptr(k), _np_ptr(v), _np_ptr(ks), _np_ptr(vs),
+                                             int(length), _stream_ptr(stream)), "zz_cache_import_fp8")
 
     def import_(self, layer: int, seq: int, kind: int, k: np.ndarray, v: np.ndarray, pos: np.ndarray,
                 length: int, stream=None) -> None:

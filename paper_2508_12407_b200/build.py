@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libzigzag_b200.so")
-SOURCES = ["zz_api.cu", "zz_append.cu", "zz_decode.cu", "zz_prefill.cu", "zz_noalloc.cu", "zz_mask.cu"]
+SOURCES = ["zz_api.cu", "zz_append.cu", "zz_decode.cu", "zz_decode_fp8.cu", "zz_prefill.cu", "zz_noalloc.cu", "zz_mask.cu"]
 
 
 def _stale() -> bool:

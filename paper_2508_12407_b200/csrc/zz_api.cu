@@ -3,6 +3,7 @@
 // checks arguments, plans launches and tracks lengths.
 #include <cuda.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cstdlib>
 #include <cstring>
@@ -66,6 +67,7 @@ struct Layout {
         off_qc, off_oc, off_dqc, off_doc, off_layer_ids, off_table, work_bytes;
     size_t arena_bytes, counters_per_layer, items_per_layer;
     long long table_entries;   // page-table entries (0: contiguous retrieval stores)
+    size_t off_desc_scratch;   // FP8 stores: [L][B] descriptors of the bf16 scratch the prefill kernel reads
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -124,6 +126,7 @@ struct zz_cache {
     std::vector<int> cap;             // [B]
     std::vector<int> len;             // [L*B] host mirror
     std::vector<SeqDesc> desc;        // [L*B]
+    std::vector<SeqDesc> desc_scratch;  // [L*B] FP8 caches: the layer's retrieval group in the bf16 scratch
     std::vector<int> layer_ids;       // exclusive retrieval layers (ascending), exclusive streaming, mixed
     int n_excl_R, n_excl_S, n_mixed;
     bool mixed_same_nR;               // every mixed layer has the same number of retrieval heads
@@ -138,6 +141,7 @@ struct zz_cache {
     bool last_nowait;   // the last launch did not wait for its predecessor: the next one must be an ordinary launch
     bool has_mixed;
     // paged retrieval stores
+    bool fp8;                         // retrieval stores hold E4M3 codes + a scale byte per token and head
     bool paged;
     int pool_pages;
     std::vector<int> free_pages;      // stack of free page ids
@@ -152,6 +156,7 @@ struct zz_cache {
     int* d_len(int l) const { return reinterpret_cast<int*>(work + lay.off_len) + (size_t)l * B; }
     int* d_pos(int l) const { return reinterpret_cast<int*>(work + lay.off_pos) + (size_t)l * B * ring; }
     SeqDesc* d_desc(int l) const { return reinterpret_cast<SeqDesc*>(work + lay.off_desc) + (size_t)l * B; }
+    SeqDesc* d_desc_scratch(int l) const { return reinterpret_cast<SeqDesc*>(work + lay.off_desc_scratch) + (size_t)l * B; }
     int* d_layer_ids() const { return reinterpret_cast<int*>(work + lay.off_layer_ids); }
     int* d_table() const { return reinterpret_cast<int*>(work + lay.off_table); }
     int* d_heads(int l) const { return reinterpret_cast<int*>(work + lay.off_heads) + (size_t)l * Hkv; }
@@ -185,6 +190,7 @@ int validate(const zz_config_t* c) {
     if (c->batch > ZZ_MAX_BATCH) return ZZ_ERR_UNSUPPORTED;
     if (c->n_q_heads % c->n_kv_heads != 0) return ZZ_ERR_UNSUPPORTED;
     if (c->n_q_heads / c->n_kv_heads > 16) return ZZ_ERR_UNSUPPORTED;
+    if (c->retrieval_kv_fp8 != 0 && c->retrieval_kv_fp8 != 1) return ZZ_ERR_INVALID_ARG;
     for (int b = 0; b < c->batch; ++b)
         if (c->capacity[b] < 1) return ZZ_ERR_INVALID_ARG;
     return ZZ_OK;
@@ -197,20 +203,24 @@ uint8_t kind_of(const zz_config_t* c, int l, int h) {
 
 // Arena: for each layer, for each sequence: retrieval group K [nR][cap][128], V likewise, then
 // streaming group K [nS][S+W][128], V likewise.  Fills `desc` if given.
-void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* desc, long long pool_pages = 0) {
+void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* desc, long long pool_pages = 0,
+                    std::vector<SeqDesc>* desc_scratch = nullptr) {
     const int L = c->n_layers, B = c->batch, Hkv = c->n_kv_heads, Hq = c->n_q_heads;
     const int ring = c->sink + c->recent;
     const int G = Hq / Hkv;
     long long off = 0;  // elements
     long long tbl = 0;  // page-table entries
     const bool paged = pool_pages > 0;
+    const bool fp8 = c->retrieval_kv_fp8 != 0;
     bool has_mixed = false;
+    int max_nR = 0;
     if (desc) desc->assign((size_t)L * B, SeqDesc());
     for (int l = 0; l < L; ++l) {
         int nR = 0;
         for (int h = 0; h < Hkv; ++h) nR += kind_of(c, l, h);
         const int nS = Hkv - nR;
         if (nR > 0 && nS > 0) has_mixed = true;
+        if (nR > max_nR) max_nR = nR;
         for (int b = 0; b < B; ++b) {
             SeqDesc d;
             d.cap = c->capacity[b];
@@ -219,6 +229,15 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
                 // retrieval rows live in the pool (offsets filled in below): entries [token block][head]
                 tbl += (long long)((d.cap + zz::kPageTokens - 1) / zz::kPageTokens) * nR;
                 d.k_off[ZZ_KIND_RETRIEVAL] = d.v_off[ZZ_KIND_RETRIEVAL] = 0;
+            } else if (fp8) {
+                // codes are one byte each (offsets count 2-byte units); the scale bytes follow the V codes
+                d.k_off[ZZ_KIND_RETRIEVAL] = off;
+                off += (long long)nR * d.cap * kD / 2;
+                d.v_off[ZZ_KIND_RETRIEVAL] = off;
+                off += (long long)nR * d.cap * kD / 2;
+                off += (long long)nR * zz::fp8_cap16(d.cap);       // K and V scale bytes: 2 * nR * cap16 bytes
+                off = (off + kD - 1) / kD * kD;                     // what follows starts on a whole bf16 row again
+                                                                    // (the prefill kernel addresses the arena by rows)
             } else {
                 d.k_off[ZZ_KIND_RETRIEVAL] = off;
                 off += (long long)nR * d.cap * kD;
@@ -242,6 +261,24 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
                 d.v_off[ZZ_KIND_RETRIEVAL] = pool_off + (long long)zz::kPageTokens * kD;
             }
     }
+    if (fp8) {
+        // bf16 scratch for one layer's retrieval rows (K then V per sequence), read by the prefill kernel
+        // when a chunk attends to rows already stored; laid out like a bf16 retrieval group
+        if (desc_scratch) desc_scratch->assign((size_t)L * B, SeqDesc());
+        long long so = off;
+        for (int b = 0; b < B; ++b) {
+            for (int l = 0; l < L && desc_scratch; ++l) {
+                int nR = 0;
+                for (int h = 0; h < Hkv; ++h) nR += kind_of(c, l, h);
+                SeqDesc d = (*desc)[(size_t)l * B + b];
+                d.k_off[ZZ_KIND_RETRIEVAL] = so;
+                d.v_off[ZZ_KIND_RETRIEVAL] = so + (long long)nR * d.cap * kD;
+                (*desc_scratch)[(size_t)l * B + b] = d;
+            }
+            so += 2LL * max_nR * c->capacity[b] * kD;
+        }
+        off = so;
+    }
     lay->table_entries = paged ? tbl : 0;
     // one spare tile of rows so that a 128-row tile read starting at the last valid row of the
     // last store stays inside the tensor map's extent (out-of-extent rows read as zero anyway)
@@ -254,6 +291,8 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
     lay->off_heads = w; w += align_up((size_t)L * Hkv * sizeof(int));
     lay->off_layer_ids = w; w += align_up((size_t)L * sizeof(int));
     lay->off_table = w; w += align_up((size_t)lay->table_entries * sizeof(int));
+    lay->off_desc_scratch = w;
+    if (fp8) w += align_up((size_t)L * B * sizeof(SeqDesc));
     // per layer: arrival counters and the split partials of the layer's launches, indexed by work
     // item (at most kMaxSlots + B * Hkv items per launch), so that the launches of different
     // layers share no scratch and may overlap
@@ -326,8 +365,9 @@ void plan_splits(const zz_cache* c, const int* n, int Hg, int* warps, int* chunk
         if (s < 1) s = 1;
         chunk[b] = (n[b] + s - 1) / s;            // equal splits inside the sequence
         if (chunk[b] < 1) chunk[b] = 1;
-        if (c->paged) {
-            // splits start at multiples of 16 tokens, so that no 16-token block straddles a page
+        if (c->paged || c->fp8) {
+            // splits start at multiples of 16 tokens, so that no 16-token block straddles a page (and the
+            // scale bytes of a block of an FP8 store are one aligned 16-byte piece)
             chunk[b] = (chunk[b] + 15) / 16 * 16;
             s = (n[b] + chunk[b] - 1) / chunk[b];
             if (s < 1) s = 1;
@@ -395,13 +435,18 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
                         const int* d_layer_ids = nullptr, int n_multi = 1) {
     const int Hg = (kind == ZZ_KIND_RETRIEVAL) ? c->nR[layer] : c->Hkv - c->nR[layer];
     if (Hg == 0) return ZZ_OK;
+    // FP8 retrieval stores: the step's token has been stored by a quantising append launched just
+    // before (quant_append_step); the kernel attends over len + 1 rows and fuses nothing
+    const bool fp8 = c->fp8 && kind == ZZ_KIND_RETRIEVAL;
+    const bool with_token = k_new != nullptr;
     zz::DecodeParams p;
     memset(&p, 0, sizeof p);
     p.arena = c->d_arena();
     p.len = c->d_len(layer);
     for (int b = 0; b < c->B; ++b) p.sd[b] = c->desc[(size_t)layer * c->B + b];
-    p.k_new = k_new;
-    p.v_new = v_new;
+    p.k_new = fp8 ? nullptr : k_new;
+    p.v_new = fp8 ? nullptr : v_new;
+    p.appended = (fp8 && with_token) ? 1 : 0;
     p.head_list = c->d_heads(layer);
     p.pos = c->d_pos(layer);
     p.seq_counters = c->d_counters(layer) + (size_t)c->B * c->Hkv;
@@ -428,7 +473,7 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
     p.page_table = c->paged ? c->d_table() : nullptr;
     int n[ZZ_MAX_BATCH];
     for (int b = 0; b < c->B; ++b) {
-        const int len = c->len[(size_t)layer * c->B + b] + (k_new ? 1 : 0);
+        const int len = c->len[(size_t)layer * c->B + b] + (with_token ? 1 : 0);
         n[b] = (kind == ZZ_KIND_RETRIEVAL) ? len : (len < c->ring ? len : c->ring);
     }
     int warps = 4;
@@ -463,8 +508,45 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
         p.st_cnt = (long long)c->lay.counters_per_layer;
         p.st_part = (long long)c->lay.items_per_layer * c->G;
     }
-    const cudaError_t e = zz::launch_decode(p, items, warps, st, overlap, n_multi);
+    const cudaError_t e = fp8 ? zz::launch_decode_fp8(p, items, warps, st, overlap, n_multi)
+                              : zz::launch_decode(p, items, warps, st, overlap, n_multi);
     zz::prof_end(pk, st);
+    return e == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
+}
+
+// FP8 caches: store (quantised) the rows a call adds to the retrieval heads.  Chunk form: one layer,
+// n_new[b] packed tokens per sequence.  Step form (n_new == nullptr): one token per sequence for
+// `n_layers` layers listed in d_layer_ids, k/v being [layer][B][Hkv][128]; the layers must have the
+// same number of retrieval heads.  The lengths stay as they are (the launch after this one moves them).
+int quant_append(zz_cache* c, int layer, const __nv_bfloat16* k, const __nv_bfloat16* v, const int32_t* n_new,
+                 const int* d_layer_ids, int n_layers, cudaStream_t st) {
+    const int nR = c->nR[layer];
+    if (nR == 0) return ZZ_OK;
+    zz::QuantAppendParams p;
+    memset(&p, 0, sizeof p);
+    p.arena = c->arena;
+    p.desc_table = c->d_desc(0);
+    p.len = c->d_len(0);
+    p.head_list = c->d_heads(0);
+    p.k_new = k;
+    p.v_new = v;
+    p.layer_ids = d_layer_ids;
+    p.status = c->d_status();
+    p.layer = layer;
+    p.nR = nR;
+    p.Hkv = c->Hkv;
+    p.B = c->B;
+    int off = 0, worst = 1;
+    for (int b = 0; b < c->B; ++b) {
+        p.n_new[b] = n_new ? n_new[b] : 1;
+        p.tok_off[b] = off;
+        off += p.n_new[b];
+        if (p.n_new[b] > worst) worst = p.n_new[b];
+    }
+    zz::prof_begin(zz::kProfAppend, st);
+    c->last_nowait = false;
+    const cudaError_t e = zz::launch_quant_append(p, worst, d_layer_ids ? n_layers : 1, st);
+    zz::prof_end(zz::kProfAppend, st);
     return e == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
 }
 
@@ -499,9 +581,29 @@ int launch_prefill_group(zz_cache* c, int layer, int kind, const CUtensorMap* tq
     const int nR = c->nR[layer];
     const int Hg = (kind == ZZ_KIND_RETRIEVAL) ? nR : c->Hkv - nR;
     if (Hg == 0) return ZZ_OK;
+    const bool fp8 = c->fp8 && kind == ZZ_KIND_RETRIEVAL;
+    if (fp8) {
+        // rows already stored are expanded to bf16 in the scratch (exactly: an FP8 value is a bf16
+        // number), and the kernel reads them there; the chunk's own K/V are attended to as given
+        int max_len = 0;
+        for (int b = 0; b < c->B; ++b) max_len = std::max(max_len, c->len[(size_t)layer * c->B + b]);
+        if (max_len > 0) {
+            zz::DequantParams dq;
+            dq.arena = c->arena;
+            dq.src = c->d_desc(layer);
+            dq.dst = c->d_desc_scratch(layer);
+            dq.len = c->d_len(layer);
+            dq.nR = nR;
+            dq.B = c->B;
+            zz::prof_begin(zz::kProfOther, st);
+            const cudaError_t de = zz::launch_dequant(dq, max_len, st);
+            zz::prof_end(zz::kProfOther, st);
+            if (de != cudaSuccess) return ZZ_ERR_CUDA;
+        }
+    }
     zz::PrefillParams p;
     memset(&p, 0, sizeof p);
-    p.desc = c->d_desc(layer);
+    p.desc = fp8 ? c->d_desc_scratch(layer) : c->d_desc(layer);
     p.len = c->d_len(layer);
     p.pos = c->d_pos(layer);
     p.out = out;
@@ -567,6 +669,7 @@ static int query_impl(const zz_config_t* cfg, long long pool_pages, size_t* aren
     const int v = validate(cfg);
     if (v != ZZ_OK) return v;
     if (!arena_bytes || !workspace_bytes) return ZZ_ERR_INVALID_ARG;
+    if (cfg->retrieval_kv_fp8 && pool_pages > 0) return ZZ_ERR_UNSUPPORTED;   // FP8 stores are contiguous
     Layout lay;
     compute_layout(cfg, &lay, nullptr, pool_pages);
     if (lay.table_entries > 0x7fffffffLL) return ZZ_ERR_UNSUPPORTED;
@@ -610,6 +713,7 @@ static int create_impl(const zz_config_t* cfg, long long pool_pages, void* d_are
     const int v = validate(cfg);
     if (v != ZZ_OK) return v;
     if (!d_arena || !d_workspace || !out) return ZZ_ERR_INVALID_ARG;
+    if (cfg->retrieval_kv_fp8 && pool_pages > 0) return ZZ_ERR_UNSUPPORTED;
     if (((uintptr_t)d_arena % kAlign) || ((uintptr_t)d_workspace % kAlign)) return ZZ_ERR_INVALID_ARG;
     zz_cache* c = new (std::nothrow) zz_cache();
     if (!c) return ZZ_ERR_INVALID_ARG;
@@ -621,7 +725,8 @@ static int create_impl(const zz_config_t* cfg, long long pool_pages, void* d_are
     c->decode_overlap = 3;
     c->last_nowait = false;
     c->decode_multi_waves = 8;
-    compute_layout(cfg, &c->lay, &c->desc, pool_pages);
+    c->fp8 = cfg->retrieval_kv_fp8 != 0;
+    compute_layout(cfg, &c->lay, &c->desc, pool_pages, &c->desc_scratch);
     if (c->lay.table_entries > 0x7fffffffLL) {
         delete c;
         return ZZ_ERR_UNSUPPORTED;
@@ -680,6 +785,7 @@ static int create_impl(const zz_config_t* cfg, long long pool_pages, void* d_are
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e == cudaSuccess) e = zz::decode_setup();
     if (e == cudaSuccess) e = zz::prefill_setup();
+    if (e == cudaSuccess && c->fp8) e = zz::decode_fp8_setup();
     if (e == cudaSuccess) e = cudaMemset(c->arena, 0, c->lay.arena_bytes);
     if (e == cudaSuccess) e = cudaMemset(c->work, 0, c->lay.off_part_ml);
     if (e == cudaSuccess) e = cudaMemset(c->work + c->lay.off_pos, 0xff, (size_t)c->L * c->B * c->ring * sizeof(int));
@@ -687,6 +793,9 @@ static int create_impl(const zz_config_t* cfg, long long pool_pages, void* d_are
         e = cudaMemset(c->work + c->lay.off_table, 0xff, (size_t)c->lay.table_entries * sizeof(int));
     if (e == cudaSuccess)
         e = cudaMemcpy(c->work + c->lay.off_desc, c->desc.data(), c->desc.size() * sizeof(SeqDesc),
+                       cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && c->fp8)
+        e = cudaMemcpy(c->work + c->lay.off_desc_scratch, c->desc_scratch.data(), c->desc_scratch.size() * sizeof(SeqDesc),
                        cudaMemcpyHostToDevice);
     if (e == cudaSuccess)
         e = cudaMemcpy(c->work + c->lay.off_heads, c->heads.data(), c->heads.size() * sizeof(int),
@@ -819,8 +928,14 @@ int zz_kv_append(zz_cache_t* c, int layer, const void* d_k, const void* d_v, con
         const int rp = reserve_pages(c, layer, layer + 1, h_n_new, static_cast<cudaStream_t>(stream));
         if (rp != ZZ_OK) return rp;
     }
+    if (c->fp8 && nR > 0) {
+        const int qr = quant_append(c, layer, static_cast<const __nv_bfloat16*>(d_k), static_cast<const __nv_bfloat16*>(d_v),
+                                    h_n_new, nullptr, 1, static_cast<cudaStream_t>(stream));
+        if (qr != ZZ_OK) return qr;
+    }
     zz::AppendParams p;
     memset(&p, 0, sizeof p);
+    p.skip_retrieval = (c->fp8 && nR > 0) ? 1 : 0;     // (the launch still moves the lengths)
     p.arena = c->d_arena();
     p.desc = c->d_desc(layer);
     p.len = c->d_len(layer);
@@ -907,6 +1022,11 @@ static int decode_step_impl(zz_cache_t* c, int layer, const void* d_q, const voi
     const __nv_bfloat16* v = static_cast<const __nv_bfloat16*>(d_v);
     __nv_bfloat16* out = static_cast<__nv_bfloat16*>(d_out);
     int r;
+    if (c->fp8 && nR > 0) {
+        r = quant_append(c, layer, k, v, nullptr, nullptr, 1, st);
+        if (r != ZZ_OK) return r;
+        overlap = 0;       // the attention launch reads what the append wrote: plain stream order or a wait at entry
+    }
     if (!c->mixed(layer)) {
         const int kind = nR ? ZZ_KIND_RETRIEVAL : ZZ_KIND_STREAMING;
         r = launch_decode_group(c, layer, kind, q, out, 0, st, k, v, 1,
@@ -968,7 +1088,12 @@ int zz_decode_step_all(zz_cache_t* c, const void* d_q, const void* d_k, const vo
         const int oS = c->n_excl_R, oM = c->n_excl_R + c->n_excl_S;
         int r = ZZ_OK;
         bool first = true;
-        if (c->n_mixed > 0) r = regroup(c, -1, q, c->d_dqc(), (long long)c->n_mixed * c->B, 1, st);
+        if (c->fp8) {
+            // the step's rows of every retrieval head, quantised into their slots before anything attends
+            if (c->n_excl_R > 0) r = quant_append(c, c->layer_ids[0], k, v, nullptr, ids, c->n_excl_R, st);
+            if (r == ZZ_OK && c->n_mixed > 0) r = quant_append(c, c->layer_ids[oM], k, v, nullptr, ids + oM, c->n_mixed, st);
+        }
+        if (r == ZZ_OK && c->n_mixed > 0) r = regroup(c, -1, q, c->d_dqc(), (long long)c->n_mixed * c->B, 1, st);
         if (r == ZZ_OK && c->n_excl_S > 0) {
             r = launch_decode_group(c, c->layer_ids[oS], ZZ_KIND_STREAMING, q, out, 0, st, k, v, 1, first ? 0 : 1,
                                     ids + oS, c->n_excl_S);
@@ -1161,6 +1286,7 @@ int zz_cache_export(zz_cache_t* c, int layer, int seq, int kind, void* h_k, void
     const int r = zz_cache_export_shape(c, layer, seq, kind, &nh, &ns);
     if (r != ZZ_OK) return r;
     if (!h_k || !h_v || !h_pos || !h_len) return ZZ_ERR_INVALID_ARG;
+    if (c->fp8 && kind == ZZ_KIND_RETRIEVAL) return ZZ_ERR_UNSUPPORTED;   // use zz_cache_export_fp8
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const SeqDesc& d = c->desc[(size_t)layer * c->B + seq];
     const size_t bytes = (size_t)nh * ns * kD * 2;
@@ -1203,6 +1329,7 @@ int zz_cache_import(zz_cache_t* c, int layer, int seq, int kind, const void* h_k
     const int r = zz_cache_export_shape(c, layer, seq, kind, &nh, &ns);
     if (r != ZZ_OK) return r;
     if (!h_k || !h_v || !h_pos || len < 0) return ZZ_ERR_INVALID_ARG;
+    if (c->fp8 && kind == ZZ_KIND_RETRIEVAL) return ZZ_ERR_UNSUPPORTED;   // use zz_cache_import_fp8
     if (kind == ZZ_KIND_RETRIEVAL && len > ns) return ZZ_ERR_CAPACITY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const SeqDesc& d = c->desc[(size_t)layer * c->B + seq];
@@ -1237,6 +1364,61 @@ int zz_cache_import(zz_cache_t* c, int layer, int seq, int kind, const void* h_k
     if (e == cudaSuccess) e = cudaMemcpyAsync(c->d_len(layer) + seq, &len, sizeof(int), cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return ZZ_ERR_CUDA;
+    c->len[(size_t)layer * c->B + seq] = len;
+    return ZZ_OK;
+}
+
+// FP8 retrieval group of (layer, seq): codes [heads][cap][128] and scale bytes [heads][cap], both ways
+static int fp8_copy(zz_cache_t* c, int layer, int seq, void* h_k, void* h_v, void* h_ks, void* h_vs, bool to_host,
+                    cudaStream_t st) {
+    const SeqDesc& d = c->desc[(size_t)layer * c->B + seq];
+    const int nh = c->nR[layer], cap = d.cap, cap16 = zz::fp8_cap16(cap);
+    unsigned char* kc = c->arena + 2 * d.k_off[ZZ_KIND_RETRIEVAL];
+    unsigned char* vc = c->arena + 2 * d.v_off[ZZ_KIND_RETRIEVAL];
+    unsigned char* ks = c->arena + zz::fp8_kscale_byte_off(d.v_off[ZZ_KIND_RETRIEVAL], nh, cap);
+    unsigned char* vs = ks + (size_t)nh * cap16;
+    const size_t cb = (size_t)nh * cap * kD;
+    const cudaMemcpyKind kd = to_host ? cudaMemcpyDeviceToHost : cudaMemcpyHostToDevice;
+    cudaError_t e = cudaSuccess;
+    if (cb) {
+        e = to_host ? cudaMemcpyAsync(h_k, kc, cb, kd, st) : cudaMemcpyAsync(kc, h_k, cb, kd, st);
+        if (e == cudaSuccess) e = to_host ? cudaMemcpyAsync(h_v, vc, cb, kd, st) : cudaMemcpyAsync(vc, h_v, cb, kd, st);
+        // scale rows are padded to a multiple of 16 on the device, packed [heads][cap] on the host
+        if (e == cudaSuccess)
+            e = to_host ? cudaMemcpy2DAsync(h_ks, cap, ks, cap16, cap, nh, kd, st) : cudaMemcpy2DAsync(ks, cap16, h_ks, cap, cap, nh, kd, st);
+        if (e == cudaSuccess)
+            e = to_host ? cudaMemcpy2DAsync(h_vs, cap, vs, cap16, cap, nh, kd, st) : cudaMemcpy2DAsync(vs, cap16, h_vs, cap, cap, nh, kd, st);
+    }
+    return e == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
+}
+
+int zz_cache_export_fp8(zz_cache_t* c, int layer, int seq, void* h_k_codes, void* h_v_codes, void* h_k_scale,
+                        void* h_v_scale, int32_t* h_len, void* stream) {
+    if (bad_layer(c, layer) || seq < 0 || seq >= c->B || !h_k_codes || !h_v_codes || !h_k_scale || !h_v_scale || !h_len)
+        return ZZ_ERR_INVALID_ARG;
+    if (!c->fp8) return ZZ_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int r = fp8_copy(c, layer, seq, h_k_codes, h_v_codes, h_k_scale, h_v_scale, true, st);
+    if (r != ZZ_OK) return r;
+    int dev_len = 0;
+    if (cudaMemcpyAsync(&dev_len, c->d_len(layer) + seq, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ZZ_ERR_CUDA;
+    *h_len = dev_len;
+    return ZZ_OK;
+}
+
+int zz_cache_import_fp8(zz_cache_t* c, int layer, int seq, const void* h_k_codes, const void* h_v_codes,
+                        const void* h_k_scale, const void* h_v_scale, int32_t len, void* stream) {
+    if (bad_layer(c, layer) || seq < 0 || seq >= c->B || !h_k_codes || !h_v_codes || !h_k_scale || !h_v_scale || len < 0)
+        return ZZ_ERR_INVALID_ARG;
+    if (!c->fp8) return ZZ_ERR_UNSUPPORTED;
+    if (c->nR[layer] > 0 && len > c->cap[seq]) return ZZ_ERR_CAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int r = fp8_copy(c, layer, seq, const_cast<void*>(h_k_codes), const_cast<void*>(h_v_codes), const_cast<void*>(h_k_scale),
+                     const_cast<void*>(h_v_scale), false, st);
+    if (r != ZZ_OK) return r;
+    if (cudaMemcpyAsync(c->d_len(layer) + seq, &len, sizeof(int), cudaMemcpyHostToDevice, st) != cudaSuccess) return ZZ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ZZ_ERR_CUDA;
     c->len[(size_t)layer * c->B + seq] = len;
     return ZZ_OK;
 }

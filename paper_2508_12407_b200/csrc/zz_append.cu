@@ -24,7 +24,7 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendParams p) {
     const int n_sink = max(0, min(p.S - P, C));          // chunk tokens that are sinks
     const int tail0 = max(n_sink, C - p.W);              // first surviving non-sink chunk token
     const int n_cand = n_sink + (C - tail0);
-    const long long workR = (long long)C * p.nR * 16;
+    const long long workR = p.skip_retrieval ? 0ll : (long long)C * p.nR * 16;
     const long long workS = (long long)n_cand * nS * 16;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx < workR + workS) {

@@ -35,6 +35,16 @@ constexpr int kDecodeSplitSlots = 128;
 constexpr int kDecodeMaxSplits = 120;
 static_assert(kDecodeMaxSplits < kDecodeSplitSlots, "the merge keeps one spare slot per row");
 
+// FP8 retrieval stores (a cache built with retrieval_kv_fp8): the group of one (layer, sequence)
+// holds, from k_off[ZZ_KIND_RETRIEVAL] (counted in 2-byte units like every offset): the K codes
+// [head][cap][128] bytes (E4M3), at v_off[...] the V codes likewise, then the K scale bytes
+// [head][cap16] and the V scale bytes [head][cap16], cap16 = cap rounded up to 16 (a scale byte e
+// stands for 2^(e - 127); one per token and head).
+__host__ __device__ inline int fp8_cap16(int cap) { return (cap + 15) & ~15; }
+__host__ __device__ inline long long fp8_kscale_byte_off(long long v_off, int n_heads, int cap) {
+    return 2 * v_off + (long long)n_heads * cap * kD;
+}
+
 constexpr int kPageTokens = 128;
 constexpr long long kPageElems = 2LL * kPageTokens * kD;   // K block, then V block
 
@@ -56,6 +66,7 @@ struct AppendParams {
     const int* head_list;    // [Hkv] source KV heads: first nR retrieval heads, then streaming
     const int* page_table;   // nullptr: contiguous retrieval stores
     int nR, Hkv, ring, S, W, B;
+    int skip_retrieval;      // the retrieval heads' rows were stored by another launch (FP8 stores)
     int n_new[ZZ_MAX_BATCH];
     int tok_off[ZZ_MAX_BATCH];
 };
@@ -88,6 +99,8 @@ struct DecodeParams {
     int n_kv_total;
     int S, W;
     int bump_len;            // this launch advances len (the last launch of a layer does)
+    int appended;            // FP8 stores: the step's token was stored by the launch before this one (the
+                             // device length does not count it yet): attend over len + 1 rows
     int gdc_wait;            // 1: wait for the previous launch before touching workspace and output;
                              // 2: wait at kernel entry; 0: never
     int split_start[ZZ_MAX_BATCH + 1];  // prefix sum of per-sequence split counts
@@ -100,6 +113,34 @@ struct DecodeParams {
     const SeqDesc* desc_table;
     const int* page_table;   // nullptr: contiguous retrieval stores
     long long st_len, st_pos, st_q, st_kv, st_cnt, st_part;
+};
+
+// Quantising append into FP8 retrieval stores: rows of the retrieval heads become E4M3 codes plus a
+// scale byte.  One layer and a packed chunk (layer_ids == nullptr: n_new / tok_off per sequence), or
+// one token per sequence for several layers at once (layer_ids: k_new / v_new are [layer][B][Hkv][128]).
+// Does not change the lengths (the launch that follows does).
+struct QuantAppendParams {
+    unsigned char* arena;
+    const SeqDesc* desc_table;   // [L][B]
+    const int* len;              // [L][B] device lengths
+    const int* head_list;        // [L][Hkv] group-ordered source KV heads (retrieval heads first)
+    const __nv_bfloat16* k_new;
+    const __nv_bfloat16* v_new;
+    const int* layer_ids;        // nullptr: the single layer `layer`
+    int* status;
+    int layer, nR, Hkv, B;
+    int n_new[ZZ_MAX_BATCH];
+    int tok_off[ZZ_MAX_BATCH];
+};
+
+// FP8 rows [0, len) of one layer's retrieval stores -> bf16 rows in a scratch region laid out like a
+// bf16 retrieval group (what the prefill kernel reads when a chunk attends to an FP8 store).
+struct DequantParams {
+    unsigned char* arena;
+    const SeqDesc* src;          // [B] of the layer
+    const SeqDesc* dst;          // [B] scratch layout
+    const int* len;              // [B]
+    int nR, B;
 };
 
 struct GatherParams {
@@ -142,6 +183,10 @@ struct PrefillParams {
 cudaError_t launch_append(const AppendParams& p, int grid_x, cudaStream_t s);
 cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStream_t s, int overlap = 0, int n_layers = 1);
 cudaError_t launch_regroup(const GatherParams& p, cudaStream_t s, int programmatic);
+cudaError_t launch_quant_append(const QuantAppendParams& p, int max_new, int n_layers, cudaStream_t s);
+cudaError_t launch_dequant(const DequantParams& p, int max_len, cudaStream_t s);
+cudaError_t launch_decode_fp8(const DecodeParams& p, int n_items, int warps, cudaStream_t s, int overlap = 0, int n_layers = 1);
+cudaError_t decode_fp8_setup();
 cudaError_t launch_reset(int* len, int* pos, int L, int B, int ring, int seq, cudaStream_t s);
 cudaError_t launch_table_update(int* table, const TableUpdate& u, cudaStream_t s);
 cudaError_t decode_setup();

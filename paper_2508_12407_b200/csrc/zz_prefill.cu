@@ -260,12 +260,16 @@ __device__ __forceinline__ float2 add2(float2 a, float2 b) {
         : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
     return d;
 }
-// 2^x for a pair of finite x on the FMA pipe instead of the MUFU: x = n + f with n = round(x)
+// 2^x for a pair of x <= ~120 on the FMA pipe instead of the MUFU: x = n + f with n = round(x)
 // (taken from the low mantissa bits of x + 1.5 * 2^23) and f in [-0.5, 0.5]; 2^f by a cubic
 // fitted to minimise the relative error on that interval (7.5e-5, far below the bf16 rounding of
 // the probabilities); n goes straight into the exponent field.
 __device__ __forceinline__ float2 exp2_poly2(float2 x) {
     const float kMagic = 12582912.f;
+    // below 2^-126 the exponent arithmetic at the end would wrap around; such probabilities are zero
+    // to the row sum and to the bf16 operand alike, so the argument is held at -126
+    x.x = fmaxf(x.x, -126.f);
+    x.y = fmaxf(x.y, -126.f);
     const float2 t = add2(x, make_float2(kMagic, kMagic));
     const float2 r = add2(t, make_float2(-kMagic, -kMagic));
     const float2 f = fma2(r, make_float2(-1.f, -1.f), x);

@@ -165,3 +165,36 @@ def test_long_prefill_sampled_rows():
     def rows(P, c):
         return [0, 1, 63, 64, 127, 128, 319, 320, 321, c // 2, c - 129, c - 128, c - 2, c - 1]
     run_prefill(2, 1, 8, 2, 64, 256, [1, 0], [[6000, 2500]], seed=70, sample_rows=rows)
+
+
+def test_scores_of_very_different_magnitude():
+    """Keys (and values) of some tokens 64 times larger or smaller than the rest: scores hundreds of
+    units apart, so most probabilities underflow.  Every exponential path must turn those into zeros
+    (the polynomial one has no hardware underflow to lean on)."""
+    import torch
+    D, Hq, Hkv, S, W, C = 128, 8, 2, 16, 48, 700
+    scale = 1.0 / np.sqrt(D)
+    w = inputs.Workload("t", 2, 1, Hq, Hkv, D, S, W, 1, 0, 0, 0, seed=909)
+    cache = binding.ZigzagCache(2, 1, Hq, Hkv, S, W, [1, 0], [2 * C + 4], C)
+    rng = np.random.default_rng(909)
+    for l, kind in enumerate([1, 0]):
+        o = OracleSeq(Hkv, D, S, W, 2 * C + 4, [kind] * Hkv)
+        for chunk in range(2):
+            q, k, v = inputs.qkv_bf16(w, l, 0, chunk * C, C)
+            sh = np.where(rng.random((C, 1, 1)) < 0.1, rng.integers(-6, 7, (C, 1, 1)), 0).astype(np.float64)
+            k = inputs.f32_to_bf16_bits((inputs.bf16_bits_to_f64(k) * np.exp2(sh)).astype(np.float32))
+            v = inputs.f32_to_bf16_bits((inputs.bf16_bits_to_f64(v) * np.exp2(-np.abs(sh))).astype(np.float32))   # outputs stay of order one
+            want = o.rows(q, chunk * C + np.arange(C), np.concatenate([o.hist.k, k]), np.concatenate([o.hist.v, v]), scale)
+            dq, dk, dv = to_dev(q), to_dev(k), to_dev(v)
+            out = torch.zeros_like(dq)
+            cache.prefill_attn(l, dq, dk, dv, out, [C])
+            cache.kv_append(l, dk, dv, [C])
+            o.append(k, v)
+            assert_close(to_bits(out), want, f"layer {l} chunk {chunk}")
+        q, k, v = inputs.qkv_bf16(w, l, 0, 2 * C, 1)
+        o.append(k, v)
+        dq = to_dev(q); out = torch.zeros_like(dq)
+        cache.decode_step(l, dq, to_dev(k), to_dev(v), out)
+        assert_close(to_bits(out), o.rows(q, [2 * C], scale=scale), f"layer {l} decode")
+    assert cache.last_status() == 0
+    cache.close()
