@@ -316,8 +316,9 @@ bool bad_layer(const zz_cache* c, int layer) { return !c || layer < 0 || layer >
 
 // Split plan of one decode launch.  Short stores: 8-warp CTAs (one per SM) that each take up to
 // 384 tokens, so a warp's chain is at most three dependent steps.  Long stores: 4-warp CTAs
-// (two per SM), all work items in one wave, every sequence cut into equal splits.
-void plan_splits(const zz_cache* c, const int* n, int Hg, int* warps, int* chunk, int* split_start, int n_multi = 1) {
+// (ctas_per_sm of them fit an SM), all work items in one wave, every sequence cut into equal splits.
+void plan_splits(const zz_cache* c, const int* n, int Hg, int* warps, int* chunk, int* split_start, int n_multi = 1,
+                 int ctas_per_sm = 2) {
     long long total = 0;
     for (int b = 0; b < c->B; ++b) total += n[b];
     split_start[0] = 0;
@@ -337,7 +338,7 @@ void plan_splits(const zz_cache* c, const int* n, int Hg, int* warps, int* chunk
         return;
     }
     *warps = 4;
-    int slots = 2 * c->num_sms < kMaxSlots ? 2 * c->num_sms : kMaxSlots;
+    int slots = ctas_per_sm * c->num_sms < kMaxSlots ? ctas_per_sm * c->num_sms : kMaxSlots;
     // a grid over several layers fills the GPU with all of them together: each layer is cut into
     // fewer, longer items (decode_multi_waves waves of CTAs over the whole grid), which spends less
     // on per-CTA ramp-up, merge and partials
@@ -477,7 +478,8 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
         n[b] = (kind == ZZ_KIND_RETRIEVAL) ? len : (len < c->ring ? len : c->ring);
     }
     int warps = 4;
-    plan_splits(c, n, Hg, &warps, p.chunk, p.split_start, d_layer_ids ? n_multi : 1);
+    // (the FP8 kernel's 4-warp CTAs fit three to an SM, the bf16 kernel's two)
+    plan_splits(c, n, Hg, &warps, p.chunk, p.split_start, d_layer_ids ? n_multi : 1, fp8 ? 3 : 2);
     const int items = p.split_start[c->B] * Hg;
     const int pk = (kind == ZZ_KIND_RETRIEVAL) ? zz::kProfDecodeR : zz::kProfDecodeS;
     zz::prof_begin(pk, st);

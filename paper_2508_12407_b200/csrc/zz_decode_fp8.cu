@@ -29,10 +29,10 @@ namespace zz {
 namespace {
 
 constexpr int kBlk = 16;                          // tokens per warp step
-constexpr int kStagesF8 = 6;
+constexpr int kStagesF8 = 4;
 constexpr int kCodeBytes = kBlk * kD;             // 2 KiB of K codes (and as much of V codes) per stage
 constexpr int kStageF8 = 2 * kCodeBytes + 128;    // + 16 K scale bytes, 16 V scale bytes, padding
-constexpr int kWarpSmemF8 = kStagesF8 * kStageF8; // 25344 B per warp: 4 warps 99 KiB (two CTAs per SM), 8 warps 198 KiB
+constexpr int kWarpSmemF8 = kStagesF8 * kStageF8; // 16896 B per warp: 4 warps 66 KiB (three CTAs per SM), 8 warps 132 KiB
 
 __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                         uint32_t b0, uint32_t b1) {
@@ -48,6 +48,13 @@ __device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_codes) {
     const unsigned short x = (unsigned short)two_codes;
     asm("cvt.rn.f16x2.e4m3x2 %0, %1;\n" : "=r"(r) : "h"(x));
     return r;
+}
+// the four codes of a 32-bit register -> two f16x2 registers (codes 0, 1 and codes 2, 3)
+__device__ __forceinline__ void e4m3x4_to_f16x2x2(uint32_t four_codes, uint32_t& lo, uint32_t& hi) {
+    asm("{\n\t.reg .b16 a, b;\n\tmov.b32 {a, b}, %2;\n\t"
+        "cvt.rn.f16x2.e4m3x2 %0, a;\n\tcvt.rn.f16x2.e4m3x2 %1, b;\n\t}"
+        : "=r"(lo), "=r"(hi)
+        : "r"(four_codes));
 }
 __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
     __half2 v = __floats2half2_rn(lo, hi);
@@ -199,8 +206,11 @@ __device__ __forceinline__ void load_block_fp8(uint32_t stage, const unsigned ch
     if (lane < 2) cp_async16(stage + 2 * kCodeBytes + lane * 16, (lane ? vs : ks) + tok0, 16);
 }
 
+// Twice the tokens per byte make this kernel bound by instruction issue rather than by HBM, and its
+// chains of dependent steps are long: twelve warps per SM (168 registers, four stages) measured 7-8 %
+// faster than eight (225 registers, six stages).
 template <bool HI, int kWarps>
-__global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_fp8_kernel(const DecodeParams p) {
+__global__ void __launch_bounds__(kWarps * 32, 12 / kWarps) decode_fp8_kernel(const DecodeParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     __shared__ int s_is_last;
 
@@ -347,12 +357,16 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_fp8_kernel(con
         for (int pc = 0; pc < 4; ++pc) {
             const int r = (lane & 7) + (((lane >> 3) & 1) << 3);
             const int c = pc * 2 + (lane >> 4);
-            uint32_t m0, m1, m2, m3;
+            uint32_t m0, m1, m2, m3, b0, b1;
             ldmatrix_x4(sk + r * kD + ((c ^ (r & 7)) << 4), m0, m1, m2, m3);
-            mma_f16(sc[0], qa[2 * pc][0], qa[2 * pc][1], qa[2 * pc][2], qa[2 * pc][3], e4m3x2_to_f16x2(m0), e4m3x2_to_f16x2(m0 >> 16));
-            mma_f16(sc[1], qa[2 * pc][0], qa[2 * pc][1], qa[2 * pc][2], qa[2 * pc][3], e4m3x2_to_f16x2(m1), e4m3x2_to_f16x2(m1 >> 16));
-            mma_f16(sc[0], qa[2 * pc + 1][0], qa[2 * pc + 1][1], qa[2 * pc + 1][2], qa[2 * pc + 1][3], e4m3x2_to_f16x2(m2), e4m3x2_to_f16x2(m2 >> 16));
-            mma_f16(sc[1], qa[2 * pc + 1][0], qa[2 * pc + 1][1], qa[2 * pc + 1][2], qa[2 * pc + 1][3], e4m3x2_to_f16x2(m3), e4m3x2_to_f16x2(m3 >> 16));
+            e4m3x4_to_f16x2x2(m0, b0, b1);
+            mma_f16(sc[0], qa[2 * pc][0], qa[2 * pc][1], qa[2 * pc][2], qa[2 * pc][3], b0, b1);
+            e4m3x4_to_f16x2x2(m1, b0, b1);
+            mma_f16(sc[1], qa[2 * pc][0], qa[2 * pc][1], qa[2 * pc][2], qa[2 * pc][3], b0, b1);
+            e4m3x4_to_f16x2x2(m2, b0, b1);
+            mma_f16(sc[0], qa[2 * pc + 1][0], qa[2 * pc + 1][1], qa[2 * pc + 1][2], qa[2 * pc + 1][3], b0, b1);
+            e4m3x4_to_f16x2x2(m3, b0, b1);
+            mma_f16(sc[1], qa[2 * pc + 1][0], qa[2 * pc + 1][1], qa[2 * pc + 1][2], qa[2 * pc + 1][3], b0, b1);
         }
 
         // the block's largest V scale: the accumulators move to it when it grows (rare after the first block)
@@ -415,12 +429,15 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_fp8_kernel(con
             const int c = pc * 2 + (lane >> 4);
             uint32_t m0, m1, m2, m3;
             ldmatrix_x4_trans(sv + r * kD + ((c ^ (r & 7)) << 4), m0, m1, m2, m3);
-            const uint32_t x0 = __byte_perm(m0, 0u, 0x3120), x1 = __byte_perm(m1, 0u, 0x3120);
-            const uint32_t x2 = __byte_perm(m2, 0u, 0x3120), x3 = __byte_perm(m3, 0u, 0x3120);
-            mma_f16(o[4 * pc + 0], pa[0], pa[1], pa[2], pa[3], e4m3x2_to_f16x2(x0), e4m3x2_to_f16x2(x1));
-            mma_f16(o[4 * pc + 1], pa[0], pa[1], pa[2], pa[3], e4m3x2_to_f16x2(x0 >> 16), e4m3x2_to_f16x2(x1 >> 16));
-            mma_f16(o[4 * pc + 2], pa[0], pa[1], pa[2], pa[3], e4m3x2_to_f16x2(x2), e4m3x2_to_f16x2(x3));
-            mma_f16(o[4 * pc + 3], pa[0], pa[1], pa[2], pa[3], e4m3x2_to_f16x2(x2 >> 16), e4m3x2_to_f16x2(x3 >> 16));
+            uint32_t e0, o0, e1, o1;
+            e4m3x4_to_f16x2x2(__byte_perm(m0, 0u, 0x3120), e0, o0);
+            e4m3x4_to_f16x2x2(__byte_perm(m1, 0u, 0x3120), e1, o1);
+            mma_f16(o[4 * pc + 0], pa[0], pa[1], pa[2], pa[3], e0, e1);
+            mma_f16(o[4 * pc + 1], pa[0], pa[1], pa[2], pa[3], o0, o1);
+            e4m3x4_to_f16x2x2(__byte_perm(m2, 0u, 0x3120), e0, o0);
+            e4m3x4_to_f16x2x2(__byte_perm(m3, 0u, 0x3120), e1, o1);
+            mma_f16(o[4 * pc + 2], pa[0], pa[1], pa[2], pa[3], e0, e1);
+            mma_f16(o[4 * pc + 3], pa[0], pa[1], pa[2], pa[3], o0, o1);
         }
         __syncwarp();
     }

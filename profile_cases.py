@@ -32,6 +32,7 @@ def main():
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--recent", type=int, default=256)
     ap.add_argument("--paged", action="store_true", help="retrieval stores in 128-token pages")
+    ap.add_argument("--kv", default="bf16", choices=["bf16", "fp8"], help="storage of the retrieval stores")
     args = ap.parse_args()
     build.build()
     binding.load()
@@ -54,7 +55,7 @@ def main():
     heads_R = int(kvk.sum()) if kvk is not None else int(sum(kinds)) * Hkv
     pool = heads_R * B * ((N + 64 + 127) // 128) if args.paged else 0
     cache = binding.ZigzagCache(L, B, Hq, Hkv, S, W, kinds, [N + 64] * B, max(B * N, B),
-                                kvhead_is_retrieval=kvk, pool_pages=pool)
+                                kvhead_is_retrieval=kvk, pool_pages=pool, kv_fp8=args.kv == "fp8")
     if args.case in ("prefill_r", "prefill_s"):
         q, k, v = randn(B * N, Hq, D), randn(B * N, Hkv, D), randn(B * N, Hkv, D)
         out = torch.empty_like(q)
