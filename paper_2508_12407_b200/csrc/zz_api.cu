@@ -89,12 +89,12 @@ EncodeTiledFn get_encode() {
     return fn;
 }
 
-// [rows][heads][128] bf16 seen as a 3-D tensor; a box is 128 rows x 1 head x 64 columns (128-byte swizzle)
-bool encode_rows3d(CUtensorMap* m, const void* base, long long rows, int heads) {
+// [rows][heads][D] bf16 seen as a 3-D tensor; a box is 128 rows x 1 head x 64 columns (128-byte swizzle)
+bool encode_rows3d(CUtensorMap* m, const void* base, long long rows, int heads, int D) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)heads, (cuuint64_t)rows};
-    cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)heads * kD * 2};
+    cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)heads, (cuuint64_t)rows};
+    cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)heads * D * 2};
     cuuint32_t box[3] = {64, 1, 128};
     cuuint32_t estr[3] = {1, 1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
@@ -102,12 +102,12 @@ bool encode_rows3d(CUtensorMap* m, const void* base, long long rows, int heads) 
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// the arena as [rows][128] bf16; a box is 128 rows x 64 columns
-bool encode_rows2d(CUtensorMap* m, const void* base, long long rows) {
+// the arena as [rows][D] bf16; a box is 128 rows x 64 columns
+bool encode_rows2d(CUtensorMap* m, const void* base, long long rows, int D) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
+    cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)D * 2};
     cuuint32_t box[2] = {64, 128};
     cuuint32_t estr[2] = {1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
@@ -118,7 +118,7 @@ bool encode_rows2d(CUtensorMap* m, const void* base, long long rows) {
 }  // namespace
 
 struct zz_cache {
-    int L, B, Hq, Hkv, G, S, W, ring, max_new;
+    int L, B, Hq, Hkv, G, D, S, W, ring, max_new;
     float scale;
     std::vector<uint8_t> kind;        // [L*Hkv]
     std::vector<int> nR;              // [L] retrieval KV heads of the layer
@@ -167,7 +167,7 @@ struct zz_cache {
         return reinterpret_cast<float*>(work + lay.off_part_ml) + (size_t)l * lay.items_per_layer * G * 2;
     }
     float* d_part_o(int l) const {
-        return reinterpret_cast<float*>(work + lay.off_part_o) + (size_t)l * lay.items_per_layer * G * kD;
+        return reinterpret_cast<float*>(work + lay.off_part_o) + (size_t)l * lay.items_per_layer * G * D;
     }
     __nv_bfloat16* d_qc() const { return reinterpret_cast<__nv_bfloat16*>(work + lay.off_qc); }
     __nv_bfloat16* d_oc() const { return reinterpret_cast<__nv_bfloat16*>(work + lay.off_oc); }
@@ -186,7 +186,8 @@ int validate(const zz_config_t* c) {
     if (c->sink < 0 || c->recent < 1) return ZZ_ERR_INVALID_ARG;
     if (c->max_new_tokens < c->batch) return ZZ_ERR_INVALID_ARG;
     if (!(c->softmax_scale > 0.f)) return ZZ_ERR_INVALID_ARG;
-    if (c->head_dim != kD) return ZZ_ERR_UNSUPPORTED;
+    if (c->head_dim != 128 && c->head_dim != 64) return ZZ_ERR_UNSUPPORTED;
+    if (c->head_dim != kD && c->retrieval_kv_fp8) return ZZ_ERR_UNSUPPORTED;      // FP8 stores: head_dim 128 only
     if (c->batch > ZZ_MAX_BATCH) return ZZ_ERR_UNSUPPORTED;
     if (c->n_q_heads % c->n_kv_heads != 0) return ZZ_ERR_UNSUPPORTED;
     if (c->n_q_heads / c->n_kv_heads > 16) return ZZ_ERR_UNSUPPORTED;
@@ -208,6 +209,7 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
     const int L = c->n_layers, B = c->batch, Hkv = c->n_kv_heads, Hq = c->n_q_heads;
     const int ring = c->sink + c->recent;
     const int G = Hq / Hkv;
+    const int Dh = c->head_dim;     // (FP8 stores exist at head_dim 128 only, where Dh == Dh)
     long long off = 0;  // elements
     long long tbl = 0;  // page-table entries
     const bool paged = pool_pages > 0;
@@ -232,22 +234,22 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
             } else if (fp8) {
                 // codes are one byte each (offsets count 2-byte units); the scale bytes follow the V codes
                 d.k_off[ZZ_KIND_RETRIEVAL] = off;
-                off += (long long)nR * d.cap * kD / 2;
+                off += (long long)nR * d.cap * Dh / 2;
                 d.v_off[ZZ_KIND_RETRIEVAL] = off;
-                off += (long long)nR * d.cap * kD / 2;
+                off += (long long)nR * d.cap * Dh / 2;
                 off += (long long)nR * zz::fp8_cap16(d.cap);       // K and V scale bytes: 2 * nR * cap16 bytes
-                off = (off + kD - 1) / kD * kD;                     // what follows starts on a whole bf16 row again
+                off = (off + Dh - 1) / Dh * Dh;                     // what follows starts on a whole bf16 row again
                                                                     // (the prefill kernel addresses the arena by rows)
             } else {
                 d.k_off[ZZ_KIND_RETRIEVAL] = off;
-                off += (long long)nR * d.cap * kD;
+                off += (long long)nR * d.cap * Dh;
                 d.v_off[ZZ_KIND_RETRIEVAL] = off;
-                off += (long long)nR * d.cap * kD;
+                off += (long long)nR * d.cap * Dh;
             }
             d.k_off[ZZ_KIND_STREAMING] = off;
-            off += (long long)nS * ring * kD;
+            off += (long long)nS * ring * Dh;
             d.v_off[ZZ_KIND_STREAMING] = off;
-            off += (long long)nS * ring * kD;
+            off += (long long)nS * ring * Dh;
             if (desc) (*desc)[(size_t)l * B + b] = d;
         }
     }
@@ -258,7 +260,7 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
         if (desc)
             for (auto& d : *desc) {
                 d.k_off[ZZ_KIND_RETRIEVAL] = pool_off;
-                d.v_off[ZZ_KIND_RETRIEVAL] = pool_off + (long long)zz::kPageTokens * kD;
+                d.v_off[ZZ_KIND_RETRIEVAL] = pool_off + (long long)zz::kPageTokens * Dh;
             }
     }
     if (fp8) {
@@ -272,17 +274,17 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
                 for (int h = 0; h < Hkv; ++h) nR += kind_of(c, l, h);
                 SeqDesc d = (*desc)[(size_t)l * B + b];
                 d.k_off[ZZ_KIND_RETRIEVAL] = so;
-                d.v_off[ZZ_KIND_RETRIEVAL] = so + (long long)nR * d.cap * kD;
+                d.v_off[ZZ_KIND_RETRIEVAL] = so + (long long)nR * d.cap * Dh;
                 (*desc_scratch)[(size_t)l * B + b] = d;
             }
-            so += 2LL * max_nR * c->capacity[b] * kD;
+            so += 2LL * max_nR * c->capacity[b] * Dh;
         }
         off = so;
     }
     lay->table_entries = paged ? tbl : 0;
     // one spare tile of rows so that a 128-row tile read starting at the last valid row of the
     // last store stays inside the tensor map's extent (out-of-extent rows read as zero anyway)
-    lay->arena_bytes = align_up((size_t)off * 2 + 128 * kD * 2);
+    lay->arena_bytes = align_up((size_t)off * 2 + 128 * Dh * 2);
     size_t w = 0;
     lay->off_status = w; w += kAlign;
     lay->off_len = w; w += align_up((size_t)L * B * sizeof(int));
@@ -300,15 +302,15 @@ void compute_layout(const zz_config_t* c, Layout* lay, std::vector<SeqDesc>* des
     lay->items_per_layer = (size_t)kMaxSlots + (size_t)B * Hkv;
     lay->off_counters = w; w += align_up((size_t)L * lay->counters_per_layer * sizeof(unsigned int));
     lay->off_part_ml = w; w += align_up((size_t)L * lay->items_per_layer * G * 2 * sizeof(float));
-    lay->off_part_o = w; w += align_up((size_t)L * lay->items_per_layer * G * kD * sizeof(float));
+    lay->off_part_o = w; w += align_up((size_t)L * lay->items_per_layer * G * Dh * sizeof(float));
     lay->off_qc = w;
-    if (has_mixed) w += align_up((size_t)c->max_new_tokens * Hq * kD * 2);
+    if (has_mixed) w += align_up((size_t)c->max_new_tokens * Hq * Dh * 2);
     lay->off_oc = w;
-    if (has_mixed) w += align_up((size_t)c->max_new_tokens * Hq * kD * 2);
+    if (has_mixed) w += align_up((size_t)c->max_new_tokens * Hq * Dh * 2);
     lay->off_dqc = w;
-    if (has_mixed) w += align_up((size_t)L * B * Hq * kD * 2);
+    if (has_mixed) w += align_up((size_t)L * B * Hq * Dh * 2);
     lay->off_doc = w;
-    if (has_mixed) w += align_up((size_t)L * B * Hq * kD * 2);
+    if (has_mixed) w += align_up((size_t)L * B * Hq * Dh * 2);
     lay->work_bytes = w;
 }
 
@@ -458,7 +460,8 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
     p.bump_len = bump_len;
     p.q = q;
     p.out = out;
-    p.q_tok_stride = (long long)c->Hq * kD;
+    p.q_tok_stride = (long long)c->Hq * c->D;
+    p.D = c->D;
     p.q_head0 = q_head0;
     p.part_o = c->d_part_o(layer);
     p.part_ml = c->d_part_ml(layer);
@@ -505,8 +508,8 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
         p.part_ml = c->d_part_ml(0);
         p.st_len = c->B;
         p.st_pos = (long long)c->B * c->ring;
-        p.st_q = (long long)c->B * c->Hq * kD;
-        p.st_kv = (long long)c->B * c->Hkv * kD;
+        p.st_q = (long long)c->B * c->Hq * c->D;
+        p.st_kv = (long long)c->B * c->Hkv * c->D;
         p.st_cnt = (long long)c->lay.counters_per_layer;
         p.st_part = (long long)c->lay.items_per_layer * c->G;
     }
@@ -560,6 +563,7 @@ int regroup(zz_cache* c, int layer, const __nv_bfloat16* src, __nv_bfloat16* dst
     g.head_list = c->d_heads(layer < 0 ? 0 : layer);
     g.Hkv = c->Hkv;
     g.G = c->G;
+    g.D = c->D;
     g.tokens = tokens;
     g.to_compact = to_compact;
     g.layer_ids = nullptr;
@@ -583,6 +587,7 @@ int launch_prefill_group(zz_cache* c, int layer, int kind, const CUtensorMap* tq
     const int nR = c->nR[layer];
     const int Hg = (kind == ZZ_KIND_RETRIEVAL) ? nR : c->Hkv - nR;
     if (Hg == 0) return ZZ_OK;
+    if (c->D != kD) return ZZ_ERR_UNSUPPORTED;   // TEMP: prefill at head_dim 64
     const bool fp8 = c->fp8 && kind == ZZ_KIND_RETRIEVAL;
     if (fp8) {
         // rows already stored are expanded to bf16 in the scratch (exactly: an FP8 value is a bf16
@@ -609,7 +614,8 @@ int launch_prefill_group(zz_cache* c, int layer, int kind, const CUtensorMap* tq
     p.len = c->d_len(layer);
     p.pos = c->d_pos(layer);
     p.out = out;
-    p.tok_stride = (long long)c->Hq * kD;
+    p.tok_stride = (long long)c->Hq * c->D;
+    p.D = c->D;
     p.head_list = c->d_heads(layer);
     p.page_table = c->paged ? c->d_table() : nullptr;
     p.status = c->d_status();
@@ -672,6 +678,7 @@ static int query_impl(const zz_config_t* cfg, long long pool_pages, size_t* aren
     if (v != ZZ_OK) return v;
     if (!arena_bytes || !workspace_bytes) return ZZ_ERR_INVALID_ARG;
     if (cfg->retrieval_kv_fp8 && pool_pages > 0) return ZZ_ERR_UNSUPPORTED;   // FP8 stores are contiguous
+    if (cfg->head_dim != kD && pool_pages > 0) return ZZ_ERR_UNSUPPORTED;     // pages hold rows of 128
     Layout lay;
     compute_layout(cfg, &lay, nullptr, pool_pages);
     if (lay.table_entries > 0x7fffffffLL) return ZZ_ERR_UNSUPPORTED;
@@ -716,10 +723,12 @@ static int create_impl(const zz_config_t* cfg, long long pool_pages, void* d_are
     if (v != ZZ_OK) return v;
     if (!d_arena || !d_workspace || !out) return ZZ_ERR_INVALID_ARG;
     if (cfg->retrieval_kv_fp8 && pool_pages > 0) return ZZ_ERR_UNSUPPORTED;
+    if (cfg->head_dim != kD && pool_pages > 0) return ZZ_ERR_UNSUPPORTED;
     if (((uintptr_t)d_arena % kAlign) || ((uintptr_t)d_workspace % kAlign)) return ZZ_ERR_INVALID_ARG;
     zz_cache* c = new (std::nothrow) zz_cache();
     if (!c) return ZZ_ERR_INVALID_ARG;
     c->L = cfg->n_layers; c->B = cfg->batch; c->Hq = cfg->n_q_heads; c->Hkv = cfg->n_kv_heads;
+    c->D = cfg->head_dim;
     c->G = c->Hq / c->Hkv; c->S = cfg->sink; c->W = cfg->recent; c->ring = c->S + c->W;
     c->max_new = cfg->max_new_tokens; c->scale = cfg->softmax_scale;
     c->decode_min_chunk = 256;
@@ -810,7 +819,7 @@ static int create_impl(const zz_config_t* cfg, long long pool_pages, void* d_are
         delete c;
         return ZZ_ERR_CUDA;
     }
-    c->have_tmap_arena = encode_rows2d(&c->tmap_arena, c->arena, (long long)(c->lay.arena_bytes / (kD * 2)));
+    c->have_tmap_arena = encode_rows2d(&c->tmap_arena, c->arena, (long long)(c->lay.arena_bytes / (c->D * 2)), c->D);
     *out = c;
     return ZZ_OK;
 }
@@ -947,14 +956,14 @@ int zz_kv_append(zz_cache_t* c, int layer, const void* d_k, const void* d_v, con
     p.v_new = static_cast<const __nv_bfloat16*>(d_v);
     p.head_list = c->d_heads(layer);
     p.page_table = c->paged ? c->d_table() : nullptr;
-    p.nR = nR; p.Hkv = c->Hkv; p.ring = c->ring; p.S = c->S; p.W = c->W; p.B = c->B;
+    p.nR = nR; p.Hkv = c->Hkv; p.ring = c->ring; p.S = c->S; p.W = c->W; p.B = c->B; p.D = c->D;
     int off = 0;
     for (int b = 0; b < c->B; ++b) {
         p.n_new[b] = h_n_new[b];
         p.tok_off[b] = off;
         off += h_n_new[b];
         const long long cand = h_n_new[b] < c->ring ? h_n_new[b] : c->ring;
-        const long long work = ((long long)h_n_new[b] * nR + cand * nS) * 16;
+        const long long work = ((long long)h_n_new[b] * nR + cand * nS) * (c->D >> 3);
         if (work > worst) worst = work;
     }
     const long long gx = (worst + 255) / 256;
@@ -1049,7 +1058,7 @@ static int decode_step_impl(zz_cache_t* c, int layer, const void* d_q, const voi
 int zz_decode_step_all(zz_cache_t* c, const void* d_q, const void* d_k, const void* d_v, void* d_out,
                        void* stream) {
     if (!c || !d_q || !d_k || !d_v || !d_out) return ZZ_ERR_INVALID_ARG;
-    const size_t qs = (size_t)c->B * c->Hq * kD * 2, ks = (size_t)c->B * c->Hkv * kD * 2;
+    const size_t qs = (size_t)c->B * c->Hq * c->D * 2, ks = (size_t)c->B * c->Hkv * c->D * 2;
     // validate every layer before launching anything
     for (int l = 0; l < c->L; ++l)
         for (int b = 0; b < c->B; ++b)
@@ -1178,14 +1187,14 @@ int zz_prefill_attn(zz_cache_t* c, int layer, const void* d_q, const void* d_k, 
     const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(d_q);
     __nv_bfloat16* out = static_cast<__nv_bfloat16*>(d_out);
     alignas(64) CUtensorMap tq, tk, tv;
-    if (!encode_rows3d(&tk, d_k, total, c->Hkv) || !encode_rows3d(&tv, d_v, total, c->Hkv)) return ZZ_ERR_CUDA;
+    if (!encode_rows3d(&tk, d_k, total, c->Hkv, c->D) || !encode_rows3d(&tv, d_v, total, c->Hkv, c->D)) return ZZ_ERR_CUDA;
     if (!c->mixed(layer)) {
-        if (!encode_rows3d(&tq, q, total, c->Hq)) return ZZ_ERR_CUDA;
+        if (!encode_rows3d(&tq, q, total, c->Hq, c->D)) return ZZ_ERR_CUDA;
         const int kind = c->nR[layer] ? ZZ_KIND_RETRIEVAL : ZZ_KIND_STREAMING;
         return launch_prefill_group(c, layer, kind, &tq, &tk, &tv, out, 0, h_n_new, st);
     }
     if (total > c->max_new) return ZZ_ERR_WORKSPACE;
-    if (!encode_rows3d(&tq, c->d_qc(), total, c->Hq)) return ZZ_ERR_CUDA;
+    if (!encode_rows3d(&tq, c->d_qc(), total, c->Hq, c->D)) return ZZ_ERR_CUDA;
     int r = regroup(c, layer, q, c->d_qc(), total, 1, st);
     if (r == ZZ_OK) r = launch_prefill_group(c, layer, ZZ_KIND_RETRIEVAL, &tq, &tk, &tv, c->d_oc(), 0, h_n_new, st);
     if (r == ZZ_OK)
@@ -1197,8 +1206,8 @@ int zz_prefill_attn(zz_cache_t* c, int layer, const void* d_q, const void* d_k, 
 
 size_t zz_stage_bytes(const zz_cache_t* c, int64_t n_tokens) {
     if (!c || n_tokens < 0) return 0;
-    const size_t qb = align_up((size_t)n_tokens * c->Hq * kD * 2);
-    const size_t kb = align_up((size_t)n_tokens * c->Hkv * kD * 2);
+    const size_t qb = align_up((size_t)n_tokens * c->Hq * c->D * 2);
+    const size_t kb = align_up((size_t)n_tokens * c->Hkv * c->D * 2);
     return 2 * qb + 2 * kb;
 }
 
@@ -1213,7 +1222,7 @@ static int run_host(zz_cache_t* c, int layer, const void* h_q, const void* h_k, 
     if (stage_bytes < zz_stage_bytes(c, total)) return ZZ_ERR_WORKSPACE;
     if ((uintptr_t)d_stage % kAlign) return ZZ_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t qbytes = (size_t)total * c->Hq * kD * 2, kbytes = (size_t)total * c->Hkv * kD * 2;
+    const size_t qbytes = (size_t)total * c->Hq * c->D * 2, kbytes = (size_t)total * c->Hkv * c->D * 2;
     const size_t qb = align_up(qbytes), kb = align_up(kbytes);
     unsigned char* s = static_cast<unsigned char*>(d_stage);
     void* dq = s; void* dk = s + qb; void* dv = s + qb + kb; void* dout = s + qb + 2 * kb;
@@ -1248,7 +1257,7 @@ int zz_decode_step_all_host(zz_cache_t* c, const void* h_q, const void* h_k, con
     if (stage_bytes < zz_stage_bytes(c, total)) return ZZ_ERR_WORKSPACE;
     if ((uintptr_t)d_stage % kAlign) return ZZ_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t qbytes = (size_t)total * c->Hq * kD * 2, kbytes = (size_t)total * c->Hkv * kD * 2;
+    const size_t qbytes = (size_t)total * c->Hq * c->D * 2, kbytes = (size_t)total * c->Hkv * c->D * 2;
     const size_t qb = align_up(qbytes), kb = align_up(kbytes);
     unsigned char* s = static_cast<unsigned char*>(d_stage);
     void* dq = s; void* dk = s + qb; void* dv = s + qb + kb; void* dout = s + qb + 2 * kb;
@@ -1291,7 +1300,7 @@ int zz_cache_export(zz_cache_t* c, int layer, int seq, int kind, void* h_k, void
     if (c->fp8 && kind == ZZ_KIND_RETRIEVAL) return ZZ_ERR_UNSUPPORTED;   // use zz_cache_export_fp8
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const SeqDesc& d = c->desc[(size_t)layer * c->B + seq];
-    const size_t bytes = (size_t)nh * ns * kD * 2;
+    const size_t bytes = (size_t)nh * ns * c->D * 2;
     cudaError_t e = cudaSuccess;
     if (bytes && c->paged && kind == ZZ_KIND_RETRIEVAL) {
         // page by page into the contiguous [head][slot][128] host layout; slots without a page are left alone
@@ -1335,7 +1344,7 @@ int zz_cache_import(zz_cache_t* c, int layer, int seq, int kind, const void* h_k
     if (kind == ZZ_KIND_RETRIEVAL && len > ns) return ZZ_ERR_CAPACITY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const SeqDesc& d = c->desc[(size_t)layer * c->B + seq];
-    const size_t bytes = (size_t)nh * ns * kD * 2;
+    const size_t bytes = (size_t)nh * ns * c->D * 2;
     cudaError_t e = cudaSuccess;
     if (bytes && c->paged && kind == ZZ_KIND_RETRIEVAL) {
         const size_t lb = (size_t)layer * c->B + seq;

@@ -6,7 +6,8 @@
 
 namespace zz {
 
-// One thread moves one 16-byte piece of a K row and the matching piece of the V row.
+// One thread moves one 16-byte piece of a K row and the matching piece of the V row (a row has
+// head_dim / 8 pieces).
 // grid = (blocks over the work of the longest sequence, batch).
 //
 // Retrieval group: every new token i goes to slot len + i.
@@ -24,24 +25,25 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendParams p) {
     const int n_sink = max(0, min(p.S - P, C));          // chunk tokens that are sinks
     const int tail0 = max(n_sink, C - p.W);              // first surviving non-sink chunk token
     const int n_cand = n_sink + (C - tail0);
-    const long long workR = p.skip_retrieval ? 0ll : (long long)C * p.nR * 16;
-    const long long workS = (long long)n_cand * nS * 16;
+    const int ppr = p.D >> 3;                            // 16-byte pieces per row
+    const long long workR = p.skip_retrieval ? 0ll : (long long)C * p.nR * ppr;
+    const long long workS = (long long)n_cand * nS * ppr;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx < workR + workS) {
         int i, hi, piece, kind;
         long long slot;
         if (idx < workR) {
             kind = ZZ_KIND_RETRIEVAL;
-            piece = (int)(idx & 15);
-            const long long r = idx >> 4;
+            piece = (int)(idx % ppr);
+            const long long r = idx / ppr;
             hi = (int)(r % p.nR);
             i = (int)(r / p.nR);
             slot = (long long)P + i;
         } else {
             kind = ZZ_KIND_STREAMING;
             const long long j = idx - workR;
-            piece = (int)(j & 15);
-            const long long r = j >> 4;
+            piece = (int)(j % ppr);
+            const long long r = j / ppr;
             hi = (int)(r % nS);
             const int c = (int)(r / nS);
             i = (c < n_sink) ? c : tail0 + (c - n_sink);
@@ -51,8 +53,8 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendParams p) {
         }
         const int src_head = p.head_list[(kind == ZZ_KIND_RETRIEVAL) ? hi : p.nR + hi];
         const long long slots_per_head = (kind == ZZ_KIND_RETRIEVAL) ? sd.cap : p.ring;
-        const long long src = ((long long)(p.tok_off[b] + i) * p.Hkv + src_head) * kD + piece * 8;
-        long long dst = ((long long)hi * slots_per_head + slot) * kD + piece * 8;
+        const long long src = ((long long)(p.tok_off[b] + i) * p.Hkv + src_head) * p.D + piece * 8;
+        long long dst = ((long long)hi * slots_per_head + slot) * p.D + piece * 8;
         if (kind == ZZ_KIND_RETRIEVAL && p.page_table) {
             // paged store: the slot's page comes from the table (K rows, then V rows, per page)
             const int page = p.page_table[sd.tbl + (int)(slot >> 7) * p.nR + hi];
@@ -112,11 +114,12 @@ __global__ void __launch_bounds__(256) regroup_kernel(const GatherParams p) {
     // kernel's tail, the data dependence is kept by waiting here before anything is read
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const long long total = p.tokens * p.Hkv * p.G * 16;
+    const int ppr = p.D >> 3;
+    const long long total = p.tokens * p.Hkv * p.G * ppr;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
-        const int piece = (int)(i & 15);
-        long long r = i >> 4;
+        const int piece = (int)(i % ppr);
+        long long r = i / ppr;
         const int g = (int)(r % p.G);
         r /= p.G;
         const int c = (int)(r % p.Hkv);   // compact KV-head index
@@ -128,8 +131,8 @@ __global__ void __launch_bounds__(256) regroup_kernel(const GatherParams p) {
             hl += (long long)layer * p.Hkv;
         }
         const int h = hl[c];              // model KV-head index
-        const long long compact = ((tok * p.Hkv + c) * p.G + g) * kD + piece * 8;
-        const long long model = ((tok * p.Hkv + h) * p.G + g) * kD + piece * 8;
+        const long long compact = ((tok * p.Hkv + c) * p.G + g) * p.D + piece * 8;
+        const long long model = ((tok * p.Hkv + h) * p.G + g) * p.D + piece * 8;
         if (p.to_compact)
             *reinterpret_cast<uint4*>(p.dst + compact) = *reinterpret_cast<const uint4*>(p.src + model);
         else
@@ -150,7 +153,7 @@ cudaError_t launch_table_update(int* table, const TableUpdate& u, cudaStream_t s
 }
 
 cudaError_t launch_regroup(const GatherParams& p, cudaStream_t s, int programmatic) {
-    const long long total = p.tokens * p.Hkv * p.G * 16;
+    const long long total = p.tokens * p.Hkv * p.G * (p.D >> 3);
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
     if (blocks < 1) blocks = 1;

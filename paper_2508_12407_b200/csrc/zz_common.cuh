@@ -10,8 +10,8 @@
 
 namespace zz {
 
-constexpr int kD = 128;            // head_dim
-constexpr int kRowBytes = kD * 2;  // one K or V row of one head
+constexpr int kD = 128;            // the usual head_dim (64 is supported by the bf16 kernels; FP8 and paged stores need 128)
+constexpr int kRowBytes = kD * 2;  // one K or V row of one head at head_dim 128
 
 // Where the stores of one (layer, sequence) live in the arena, in bf16 elements from the
 // arena base.  Index [ZZ_KIND_STREAMING] is the ring group, [ZZ_KIND_RETRIEVAL] the
@@ -66,6 +66,7 @@ struct AppendParams {
     const int* head_list;    // [Hkv] source KV heads: first nR retrieval heads, then streaming
     const int* page_table;   // nullptr: contiguous retrieval stores
     int nR, Hkv, ring, S, W, B;
+    int D;                   // head_dim (64 or 128)
     int skip_retrieval;      // the retrieval heads' rows were stored by another launch (FP8 stores)
     int n_new[ZZ_MAX_BATCH];
     int tok_off[ZZ_MAX_BATCH];
@@ -84,6 +85,7 @@ struct DecodeParams {
     int* status;
     int kind;                // which group of the layer
     int ring;                // S+W
+    int D;                   // head_dim (selects the kernel instantiation)
     int Hg, G, B;
     int max_splits;          // most splits any sequence of this launch has (<= kDecodeMaxSplits); the kernel
                              // refuses a plan beyond it instead of overrunning its merge rows
@@ -149,6 +151,7 @@ struct GatherParams {
     __nv_bfloat16* dst;
     const int* head_list;    // [Hkv] group-ordered KV heads
     int Hkv, G;
+    int D;                   // head_dim
     long long tokens;
     int to_compact;          // 1: model order -> compact (gather); 0: compact -> model order (scatter)
     // several layers in one launch (decode step): token t belongs to layer layer_ids[t / toks_per_layer];
@@ -171,6 +174,7 @@ struct PrefillParams {
     int q_head0;             // first query head of the group inside a q/out row
     int n_kv_total;          // KV heads per row of the chunk K/V
     int ring, S, W, Hg, G, B;
+    int D;                   // head_dim (selects the kernel instantiation)
     int total_tiles;         // 128-row query tiles over the whole batch
     int n_items;             // work items of the launch (set by the launcher)
     float scale_log2;

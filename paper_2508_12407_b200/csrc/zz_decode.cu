@@ -29,9 +29,7 @@ namespace zz {
 namespace {
 
 constexpr int kBlk = 16;                       // tokens per warp step
-constexpr int kStages = 3;
-constexpr int kStageBytes = kBlk * kRowBytes;  // 4 KiB of K (and as much of V) per stage
-constexpr int kWarpSmem = kStages * 2 * kStageBytes;   // 24 KiB per warp
+constexpr int kWarpSmem = 24 * 1024;           // per warp: 3 stages of 2 x 4 KiB at head_dim 128, 6 stages of 2 x 2 KiB at 64
 // 4 warps: 96 KiB, two CTAs per SM (long contexts); 8 warps: 192 KiB, one CTA per SM (short
 // stores, where the per-warp chain of dependent steps is what costs)
 
@@ -39,24 +37,48 @@ constexpr int kWarpSmem = kStages * 2 * kStageBytes;   // 24 KiB per warp
 // Row r, 16-byte piece c lands at r*256 + ((c ^ (r & 7)) * 16): conflict-free for ldmatrix.
 // Slot `new_slot` (if inside the block) is the token being appended by this very launch: its
 // row comes from the caller's k_new/v_new instead of the store.
+template <int HD>
 __device__ __forceinline__ void load_block(uint32_t stage_k, uint32_t stage_v, const __nv_bfloat16* kbase,
                                            const __nv_bfloat16* vbase, int tok0, int tok_end, int lane,
                                            int new_slot, const __nv_bfloat16* knew, const __nv_bfloat16* vnew,
                                            uint64_t policy) {
+    constexpr int kRowB = HD * 2;              // bytes of a row
+    constexpr int kPieces = HD / 8;            // 16-byte pieces of a row
+    if (HD == 64) {
+        // 128-byte rows: lane -> (row it * 4 + lane / 8, piece lane % 8), pieces XOR-swizzled by row
+        const bool whole = tok0 + kBlk <= tok_end && (new_slot < tok0 || new_slot >= tok0 + kBlk);
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int r = it * 4 + (lane >> 3), c = lane & 7;
+            const int tok = tok0 + r;
+            const int ok = tok < tok_end;
+            const long long off = (long long)(ok ? tok : tok0) * HD + c * 8;
+            const uint32_t so = r * kRowB + ((c ^ (r & 7)) << 4);
+            if (whole) {
+                cp_async16_full(stage_k + so, kbase + off, policy);
+                cp_async16_full(stage_v + so, vbase + off, policy);
+            } else {
+                const bool fresh = tok == new_slot;
+                cp_async16(stage_k + so, fresh ? knew + c * 8 : kbase + off, ok ? 16 : 0);
+                cp_async16(stage_v + so, fresh ? vnew + c * 8 : vbase + off, ok ? 16 : 0);
+            }
+        }
+        return;
+    }
     if (tok0 + kBlk <= tok_end && (new_slot < tok0 || new_slot >= tok0 + kBlk)) {
         // Whole block from the store (all but the edge blocks of a range): one pointer per lane, every
         // further address a constant away.  Row r = 2*it + r0 swizzles with (r & 7) = 2*(it & 3) + r0,
         // which touches bits the two terms do not share, so it folds into one XOR per iteration.
         const int r0 = lane >> 4, c = lane & 15;
-        const long long off0 = (long long)(tok0 + r0) * kD + c * 8;
+        const long long off0 = (long long)(tok0 + r0) * HD + c * 8;
         const __nv_bfloat16* kp = kbase + off0;
         const __nv_bfloat16* vp = vbase + off0;
-        const uint32_t so0 = r0 * kRowBytes + ((c ^ r0) << 4);
+        const uint32_t so0 = r0 * kRowB + ((c ^ r0) << 4);
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
-            const uint32_t so = (so0 ^ ((it & 3) << 5)) + it * 2 * kRowBytes;
-            cp_async16_full(stage_k + so, kp + it * 2 * kD, policy);
-            cp_async16_full(stage_v + so, vp + it * 2 * kD, policy);
+            const uint32_t so = (so0 ^ ((it & 3) << 5)) + it * 2 * kRowB;
+            cp_async16_full(stage_k + so, kp + it * 2 * HD, policy);
+            cp_async16_full(stage_v + so, vp + it * 2 * HD, policy);
         }
         return;
     }
@@ -66,8 +88,8 @@ __device__ __forceinline__ void load_block(uint32_t stage_k, uint32_t stage_v, c
         const int r = idx >> 4, c = idx & 15;
         const int tok = tok0 + r;
         const int ok = tok < tok_end;
-        const long long off = (long long)(ok ? tok : tok0) * kD + c * 8;
-        const uint32_t so = r * kRowBytes + ((c ^ (r & 7)) << 4);
+        const long long off = (long long)(ok ? tok : tok0) * HD + c * 8;
+        const uint32_t so = r * kRowB + ((c ^ (r & 7)) << 4);
         const bool fresh = tok == new_slot;
         cp_async16(stage_k + so, fresh ? knew + c * 8 : kbase + off, ok ? 16 : 0);
         cp_async16(stage_v + so, fresh ? vnew + c * 8 : vbase + off, ok ? 16 : 0);
@@ -76,8 +98,13 @@ __device__ __forceinline__ void load_block(uint32_t stage_k, uint32_t stage_v, c
 
 // HI = group size above 8 (rows 8..15 of the tile carry query heads too).
 // kPaged: the retrieval store is paged (compiled apart, so that the contiguous kernel carries none of it).
-template <bool HI, int kWarps, bool kPaged>
+// HD = head_dim (128, or 64: half the row bytes, twice the stages, half the MMA steps and accumulators).
+template <bool HI, int kWarps, bool kPaged, int HD>
 __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const DecodeParams p) {
+    constexpr int kRowB = HD * 2;                          // bytes of a K or V row
+    constexpr int kStageBytes = kBlk * kRowB;              // K (and as much of V) per stage
+    constexpr int kStages = kWarpSmem / (2 * kStageBytes); // 3 at head_dim 128, 6 at 64: the same bytes in flight
+    constexpr int kKSteps = HD / 16;                       // 16-dim MMA steps of Q K^T, 16-column pairs of P V
     extern __shared__ __align__(1024) unsigned char smem[];
     __shared__ int s_is_last;
 
@@ -103,7 +130,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     const int* const head_list_p = p.head_list + (long long)li * p.n_kv_total;
     unsigned int* const counters_p = p.counters + (long long)li * p.st_cnt;
     unsigned int* const seq_counters_p = p.seq_counters + (long long)li * p.st_cnt;
-    float* const part_o_p = p.part_o + (long long)li * p.st_part * kD;
+    float* const part_o_p = p.part_o + (long long)li * p.st_part * HD;
     float* const part_ml_p = p.part_ml + (long long)li * p.st_part * 2;
 
     // ---- which work item -----------------------------------------------------------
@@ -130,8 +157,8 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     const long long slots_per_head = (p.kind == ZZ_KIND_RETRIEVAL) ? sd.cap : p.ring;
     // paged retrieval store: the bases are the pool's; each 16-token block adds its page's offset
     constexpr bool paged = kPaged;
-    __nv_bfloat16* kbase = p.arena + sd.k_off[p.kind] + (paged ? 0ll : (long long)hg * slots_per_head * kD);
-    __nv_bfloat16* vbase = p.arena + sd.v_off[p.kind] + (paged ? 0ll : (long long)hg * slots_per_head * kD);
+    __nv_bfloat16* kbase = p.arena + sd.k_off[p.kind] + (paged ? 0ll : (long long)hg * slots_per_head * HD);
+    __nv_bfloat16* vbase = p.arena + sd.v_off[p.kind] + (paged ? 0ll : (long long)hg * slots_per_head * HD);
     const int* const tbl = paged ? p.page_table + sd.tbl + hg : nullptr;   // entry of page g: tbl[g * Hg]
     int new_slot = -1;
     const __nv_bfloat16* knew = nullptr;
@@ -151,7 +178,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     if (fused) {
         const int t = len_old;
         new_slot = (p.kind == ZZ_KIND_RETRIEVAL || t < p.S) ? t : p.S + ((t - p.S) % p.W);
-        const long long src = ((long long)b * p.n_kv_total + head_list_p[p.kv_head0 + hg]) * kD;
+        const long long src = ((long long)b * p.n_kv_total + head_list_p[p.kv_head0 + hg]) * HD;
         knew = k_new_p + src;
         vnew = v_new_p + src;
     }
@@ -165,26 +192,26 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     if (fused && new_slot >= s0 && new_slot < s1 && warp == kWarps - 1) {
         const int c = lane & 15;
         const __nv_bfloat16* src = (lane < 16 ? knew : vnew) + c * 8;
-        long long slot_off = (long long)new_slot * kD;
+        long long slot_off = (long long)new_slot * HD;
         if (paged)
-            slot_off = (long long)tbl[(new_slot >> 7) * p.Hg] * kPageElems + (new_slot & (kPageTokens - 1)) * kD;
+            slot_off = (long long)tbl[(new_slot >> 7) * p.Hg] * kPageElems + (new_slot & (kPageTokens - 1)) * HD;
         __nv_bfloat16* dst = (lane < 16 ? kbase : vbase) + slot_off + c * 8;
-        *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+        if (c < HD / 8) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);   // a row has HD / 8 pieces
         if (p.kind == ZZ_KIND_STREAMING && hg == 0 && lane == 0) pos_p[(long long)b * p.ring + new_slot] = len_old;
     }
 
     // ---- query fragments: rows = the G heads of this KV head ---------------------------
     const int G = p.G;
-    const __nv_bfloat16* qb = q_p + ((long long)b * p.q_tok_stride) + (long long)(p.q_head0 + hg * G) * kD;
-    uint32_t qa[8][4];
+    const __nv_bfloat16* qb = q_p + ((long long)b * p.q_tok_stride) + (long long)(p.q_head0 + hg * G) * HD;
+    uint32_t qa[kKSteps][4];
 #pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
+    for (int kk = 0; kk < kKSteps; ++kk) {
         const int d0 = kk * 16 + tig * 2;
-        qa[kk][0] = (grp < G) ? *reinterpret_cast<const uint32_t*>(qb + grp * kD + d0) : 0u;
-        qa[kk][2] = (grp < G) ? *reinterpret_cast<const uint32_t*>(qb + grp * kD + d0 + 8) : 0u;
+        qa[kk][0] = (grp < G) ? *reinterpret_cast<const uint32_t*>(qb + grp * HD + d0) : 0u;
+        qa[kk][2] = (grp < G) ? *reinterpret_cast<const uint32_t*>(qb + grp * HD + d0 + 8) : 0u;
         if (HI) {
-            qa[kk][1] = (grp + 8 < G) ? *reinterpret_cast<const uint32_t*>(qb + (grp + 8) * kD + d0) : 0u;
-            qa[kk][3] = (grp + 8 < G) ? *reinterpret_cast<const uint32_t*>(qb + (grp + 8) * kD + d0 + 8) : 0u;
+            qa[kk][1] = (grp + 8 < G) ? *reinterpret_cast<const uint32_t*>(qb + (grp + 8) * HD + d0) : 0u;
+            qa[kk][3] = (grp + 8 < G) ? *reinterpret_cast<const uint32_t*>(qb + (grp + 8) * HD + d0 + 8) : 0u;
         } else {
             qa[kk][1] = 0u;
             qa[kk][3] = 0u;
@@ -193,9 +220,9 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
 
     // ---- per-warp state ------------------------------------------------------------------
     constexpr int NR = HI ? 2 : 1;       // row halves carried
-    float o[16][4];
+    float o[HD / 8][4];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+    for (int i = 0; i < HD / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
     float m_run[2] = {-INFINITY, -INFINITY};
     float l_run[2] = {0.f, 0.f};
 
@@ -224,7 +251,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
             win = (pg0 + lane < n_pages) ? tbl[(pg0 + lane) * p.Hg] : 0;
         }
         const int page = __shfl_sync(0xffffffffu, win, pg - pg0);
-        return (long long)page * kPageElems - (long long)pg * kPageTokens * kD;
+        return (long long)page * kPageElems - (long long)pg * kPageTokens * HD;
     };
 
     // prologue: fill kStages-1 stages
@@ -233,7 +260,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
         if (s < my_blocks) {
             const int tok0 = s0 + (warp + s * kWarps) * kBlk;
             const long long po = page_off(tok0);
-            load_block(wbase + s * 2 * kStageBytes, wbase + s * 2 * kStageBytes + kStageBytes, kbase + po, vbase + po,
+            load_block<HD>(wbase + s * 2 * kStageBytes, wbase + s * 2 * kStageBytes + kStageBytes, kbase + po, vbase + po,
                        tok0, s1, lane, new_slot, knew, vnew, l2_policy);
         }
         cp_async_commit();
@@ -246,7 +273,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
                 const int st = nx % kStages;
                 const int tok0 = s0 + (warp + nx * kWarps) * kBlk;
                 const long long po = page_off(tok0);
-                load_block(wbase + st * 2 * kStageBytes, wbase + st * 2 * kStageBytes + kStageBytes, kbase + po,
+                load_block<HD>(wbase + st * 2 * kStageBytes, wbase + st * 2 * kStageBytes + kStageBytes, kbase + po,
                            vbase + po, tok0, s1, lane, new_slot, knew, vnew, l2_policy);
             }
             cp_async_commit();
@@ -264,11 +291,11 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
 #pragma unroll
         for (int i = 0; i < 2; ++i) { sc[i][0] = sc[i][1] = sc[i][2] = sc[i][3] = 0.f; }
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
+        for (int kk = 0; kk < kKSteps; ++kk) {
             const int r = (lane & 7) + ((lane >> 4) << 3);
             const int c = kk * 2 + ((lane >> 3) & 1);
             uint32_t b0, b1, b2, b3;
-            ldmatrix_x4(sk + r * kRowBytes + ((c ^ (r & 7)) << 4), b0, b1, b2, b3);
+            ldmatrix_x4(sk + r * kRowB + ((c ^ (r & 7)) << 4), b0, b1, b2, b3);
             mma_bf16(sc[0], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b0, b1);
             mma_bf16(sc[1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b2, b3);
         }
@@ -309,7 +336,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
                 const float alpha = fast_exp2(m_run[hf] - m_new);  // 0 on the first block
                 l_run[hf] = l_run[hf] * alpha + ps;
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
+                for (int i = 0; i < HD / 8; ++i) {
                     o[i][hf * 2 + 0] *= alpha;
                     o[i][hf * 2 + 1] *= alpha;
                 }
@@ -324,11 +351,11 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
 
         // O += P V
 #pragma unroll
-        for (int nn = 0; nn < 8; ++nn) {
+        for (int nn = 0; nn < kKSteps; ++nn) {
             const int r = (lane & 7) + (((lane >> 3) & 1) << 3);
             const int c = nn * 2 + (lane >> 4);
             uint32_t b0, b1, b2, b3;
-            ldmatrix_x4_trans(sv + r * kRowBytes + ((c ^ (r & 7)) << 4), b0, b1, b2, b3);
+            ldmatrix_x4_trans(sv + r * kRowB + ((c ^ (r & 7)) << 4), b0, b1, b2, b3);
             mma_bf16(o[2 * nn], pa[0], pa[1], pa[2], pa[3], b0, b1);
             mma_bf16(o[2 * nn + 1], pa[0], pa[1], pa[2], pa[3], b2, b3);
         }
@@ -338,27 +365,31 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     // everything up to here read only this layer's stores, lengths and the caller's q/k/v
     if (p.gdc_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    finish_item<kWarps, NR, ColsBf16>(p, smem, &s_is_last, o, m_run, l_run, item, b, hg, nsplit, len_old,
+    finish_item<kWarps, NR, ColsBf16, HD>(p, smem, &s_is_last, o, m_run, l_run, item, b, hg, nsplit, len_old,
                                       fused && p.bump_len, len_p, out_p, part_o_p, part_ml_p, counters_p, seq_counters_p);
 }
 
 }  // namespace
 
-template <bool HI, int kWarps, bool kPaged>
+template <bool HI, int kWarps, bool kPaged, int HD>
 static cudaError_t setup_one() {
-    return cudaFuncSetAttribute(decode_kernel<HI, kWarps, kPaged>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(decode_kernel<HI, kWarps, kPaged, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 kWarps * kWarpSmem);
 }
 
 cudaError_t decode_setup() {
-    cudaError_t e = setup_one<false, 4, false>();
-    if (e == cudaSuccess) e = setup_one<true, 4, false>();
-    if (e == cudaSuccess) e = setup_one<false, 8, false>();
-    if (e == cudaSuccess) e = setup_one<true, 8, false>();
-    if (e == cudaSuccess) e = setup_one<false, 4, true>();
-    if (e == cudaSuccess) e = setup_one<true, 4, true>();
-    if (e == cudaSuccess) e = setup_one<false, 8, true>();
-    if (e == cudaSuccess) e = setup_one<true, 8, true>();
+    cudaError_t e = setup_one<false, 4, false, 128>();
+    if (e == cudaSuccess) e = setup_one<true, 4, false, 128>();
+    if (e == cudaSuccess) e = setup_one<false, 8, false, 128>();
+    if (e == cudaSuccess) e = setup_one<true, 8, false, 128>();
+    if (e == cudaSuccess) e = setup_one<false, 4, true, 128>();
+    if (e == cudaSuccess) e = setup_one<true, 4, true, 128>();
+    if (e == cudaSuccess) e = setup_one<false, 8, true, 128>();
+    if (e == cudaSuccess) e = setup_one<true, 8, true, 128>();
+    if (e == cudaSuccess) e = setup_one<false, 4, false, 64>();
+    if (e == cudaSuccess) e = setup_one<true, 4, false, 64>();
+    if (e == cudaSuccess) e = setup_one<false, 8, false, 64>();
+    if (e == cudaSuccess) e = setup_one<true, 8, false, 64>();
     return e;
 }
 
@@ -387,8 +418,13 @@ cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStr
     const bool hi = p.G > 8;
     cudaError_t e;
     if (warps != 4 && warps != 8) return cudaErrorInvalidValue;
-#define ZZ_LAUNCH(HI_, W_, PG_) e = cudaLaunchKernelEx(&cfg, decode_kernel<HI_, W_, PG_>, pp)
-    if (warps == 8) {
+    if (p.D != 128 && (p.D != 64 || paged)) return cudaErrorInvalidValue;   // paged stores: head_dim 128 only
+#define ZZ_LAUNCH(HI_, W_, PG_) e = cudaLaunchKernelEx(&cfg, decode_kernel<HI_, W_, PG_, 128>, pp)
+#define ZZ_LAUNCH64(HI_, W_) e = cudaLaunchKernelEx(&cfg, decode_kernel<HI_, W_, false, 64>, pp)
+    if (p.D == 64) {
+        if (warps == 8) { if (hi) ZZ_LAUNCH64(true, 8); else ZZ_LAUNCH64(false, 8); }
+        else { if (hi) ZZ_LAUNCH64(true, 4); else ZZ_LAUNCH64(false, 4); }
+    } else if (warps == 8) {
         if (paged) { if (hi) ZZ_LAUNCH(true, 8, true); else ZZ_LAUNCH(false, 8, true); }
         else { if (hi) ZZ_LAUNCH(true, 8, false); else ZZ_LAUNCH(false, 8, false); }
     } else {
@@ -396,6 +432,7 @@ cudaError_t launch_decode(const DecodeParams& p, int n_items, int warps, cudaStr
         else { if (hi) ZZ_LAUNCH(true, 4, false); else ZZ_LAUNCH(false, 4, false); }
     }
 #undef ZZ_LAUNCH
+#undef ZZ_LAUNCH64
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -76,9 +76,9 @@ struct ColsFp8 {
 
 // Everything after a CTA's main loop.  `advance_len`: this launch makes the sequence one token longer
 // (the append fused into it, or the quantising append that ran just before it) and is the layer's last.
-template <int kWarps, int NR, class Cols>
+template <int kWarps, int NR, class Cols, int HD = kD>
 __device__ __forceinline__ void finish_item(const DecodeParams& p, unsigned char* smem, int* s_is_last_p,
-                                            float (&o)[16][4], float (&m_run)[2], float (&l_run)[2], int item,
+                                            float (&o)[HD / 8][4], float (&m_run)[2], float (&l_run)[2], int item,
                                             int b, int hg, int nsplit, int len_old, bool advance_len,
                                             int* len_p, __nv_bfloat16* out_p, float* part_o_p, float* part_ml_p,
                                             unsigned int* counters_p, unsigned int* seq_counters_p) {
@@ -94,19 +94,19 @@ __device__ __forceinline__ void finish_item(const DecodeParams& p, unsigned char
     }
     __syncthreads();   // every warp is done with its pipeline memory
     float* sm_o = reinterpret_cast<float*>(smem);                  // [kWarps][16][128]
-    float* sm_ml = sm_o + kWarps * 16 * kD;                        // [kWarps][16][2]
+    float* sm_ml = sm_o + kWarps * 16 * HD;                        // [kWarps][16][2]
 #pragma unroll
     for (int hf = 0; hf < NR; ++hf) {
         const int row = grp + hf * 8;
         if (row < G) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
+            for (int i = 0; i < HD / 8; ++i) {
                 if constexpr (Cols::kAdjacent) {
-                    *reinterpret_cast<float2*>(sm_o + (warp * 16 + row) * kD + Cols::col(i, tig, 0)) =
+                    *reinterpret_cast<float2*>(sm_o + (warp * 16 + row) * HD + Cols::col(i, tig, 0)) =
                         make_float2(o[i][hf * 2], o[i][hf * 2 + 1]);
                 } else {
-                    sm_o[(warp * 16 + row) * kD + Cols::col(i, tig, 0)] = o[i][hf * 2];
-                    sm_o[(warp * 16 + row) * kD + Cols::col(i, tig, 1)] = o[i][hf * 2 + 1];
+                    sm_o[(warp * 16 + row) * HD + Cols::col(i, tig, 0)] = o[i][hf * 2];
+                    sm_o[(warp * 16 + row) * HD + Cols::col(i, tig, 1)] = o[i][hf * 2 + 1];
                 }
             }
             if (tig == 0) {
@@ -118,9 +118,9 @@ __device__ __forceinline__ void finish_item(const DecodeParams& p, unsigned char
     __syncthreads();
 
     const long long pair = (long long)b * p.Hg + hg;
-    __nv_bfloat16* outb = out_p + ((long long)b * p.q_tok_stride) + (long long)(p.q_head0 + hg * G) * kD;
-    for (int idx = threadIdx.x; idx < G * kD; idx += kWarps * 32) {
-        const int row = idx >> 7, d = idx & 127;
+    __nv_bfloat16* outb = out_p + ((long long)b * p.q_tok_stride) + (long long)(p.q_head0 + hg * G) * HD;
+    for (int idx = threadIdx.x; idx < G * HD; idx += kWarps * 32) {
+        const int row = idx / HD, d = idx % HD;
         float M = -INFINITY;
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) M = fmaxf(M, sm_ml[(w * 16 + row) * 2]);
@@ -130,13 +130,13 @@ __device__ __forceinline__ void finish_item(const DecodeParams& p, unsigned char
             const float mw = sm_ml[(w * 16 + row) * 2];
             const float f = (mw == -INFINITY) ? 0.f : fast_exp2(mw - M);
             L += f * sm_ml[(w * 16 + row) * 2 + 1];
-            acc += f * sm_o[(w * 16 + row) * kD + d];
+            acc += f * sm_o[(w * 16 + row) * HD + d];
         }
         if (nsplit == 1) {
-            outb[row * kD + d] = __float2bfloat16_rn(acc / L);
+            outb[row * HD + d] = __float2bfloat16_rn(acc / L);
         } else {
             const long long po = (long long)item * G + row;   // partials are indexed by work item
-            part_o_p[po * kD + d] = acc;
+            part_o_p[po * HD + d] = acc;
             if (d == 0) {
                 part_ml_p[po * 2 + 0] = M;
                 part_ml_p[po * 2 + 1] = L;
@@ -175,12 +175,12 @@ __device__ __forceinline__ void finish_item(const DecodeParams& p, unsigned char
     float* sm_f = sm_m + 16 * kMaxSplitsSmem;                // [16][128] sum, then factor
     constexpr int kRound = 40;                               // splits whose partials are held at once (one round for the usual 37 of a 32K store)
     for (int row0 = 0; row0 < G; row0 += kWarps) {
-        const int row = row0 + warp;                         // this warp's row (4 dims per lane)
-        const bool row_ok = row < G;
+        const int row = row0 + warp;                         // this warp's row (4 dims per lane; half the lanes at head_dim 64)
+        const bool row_ok = row < G && lane * 4 < HD;
         // split s of this (sequence, head) is work item item0 + s * Hg
         const long long item0 = (long long)p.split_start[b] * p.Hg + hg;
-        const float* pbase = part_o_p + (item0 * G + (row_ok ? row : 0)) * kD + lane * 4;
-        const long long sstride = (long long)p.Hg * G * kD;
+        const float* pbase = part_o_p + (item0 * G + (row_ok ? row : 0)) * HD + lane * 4;
+        const long long sstride = (long long)p.Hg * G * HD;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int sb = 0; sb < nsplit; sb += kRound) {
             float4 v[kRound];
@@ -199,7 +199,7 @@ __device__ __forceinline__ void finish_item(const DecodeParams& p, unsigned char
                     }
                 }
                 __syncthreads();
-                if (row_ok) {
+                if (row < G) {
                     float M = -INFINITY;
                     for (int s = lane; s < nsplit; s += 32) M = fmaxf(M, sm_m[row * kMaxSplitsSmem + s]);
 #pragma unroll
@@ -230,7 +230,7 @@ __device__ __forceinline__ void finish_item(const DecodeParams& p, unsigned char
             uint2 w;
             w.x = pack_bf16(acc.x * inv, acc.y * inv);
             w.y = pack_bf16(acc.z * inv, acc.w * inv);
-            *reinterpret_cast<uint2*>(outb + row * kD + lane * 4) = w;
+            *reinterpret_cast<uint2*>(outb + row * HD + lane * 4) = w;
         }
         __syncthreads();
     }

@@ -95,6 +95,7 @@ extern "C" int zz_decode_attn_static(const void* d_q, const void* d_k, const voi
     p.seq_counters = p.counters + (size_t)batch * n_kv_heads;
     p.status = reinterpret_cast<int*>(scratch + kOffStatus);
     p.kind = ZZ_KIND_RETRIEVAL;
+    p.D = zz::kD;
     p.ring = 1;
     p.Hg = n_kv_heads;
     p.G = G;

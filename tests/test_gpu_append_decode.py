@@ -15,9 +15,9 @@ def _built():
     binding.load()
 
 
-def make(L, B, Hq, Hkv, S, W, kinds, cap, kvk=None, max_new=4096, pool_pages=0):
+def make(L, B, Hq, Hkv, S, W, kinds, cap, kvk=None, max_new=4096, pool_pages=0, D=128):
     return binding.ZigzagCache(L, B, Hq, Hkv, S, W, kinds, cap, max_new, kvhead_is_retrieval=kvk,
-                               pool_pages=pool_pages)
+                               pool_pages=pool_pages, head_dim=D)
 
 
 def layer_kv_kinds(kinds, Hkv, kvk, l):
@@ -27,11 +27,10 @@ def layer_kv_kinds(kinds, Hkv, kvk, l):
 
 
 def run_append_decode(L, B, Hq, Hkv, S, W, kinds, lens, n_decode, seed, kvk=None, chunk_cap=300,
-                      check_every=1, pool_pages=0, tune=None):
-    D = 128
+                      check_every=1, pool_pages=0, tune=None, D=128):
     scale = 1.0 / np.sqrt(D)
     cap = [int(n) + n_decode for n in lens]
-    cache = make(L, B, Hq, Hkv, S, W, kinds, cap, kvk, max_new=max(4096, chunk_cap * B), pool_pages=pool_pages)
+    cache = make(L, B, Hq, Hkv, S, W, kinds, cap, kvk, max_new=max(4096, chunk_cap * B), pool_pages=pool_pages, D=D)
     for key, value in (tune or {}).items():
         cache.tune(key, value)
     w = inputs.Workload("t", L, B, Hq, Hkv, D, S, W, int(sum(kinds)), 0, 0, n_decode, seed=seed)
@@ -136,6 +135,23 @@ def test_short_plan_threshold_tuned_up(short, n):
     # 137 splits of 512 tokens would overrun the merge rows (long plan instead); 98 splits of 1024
     # tokens is a legal short plan with many splits; 127 of 1024 is again past the limit
     run_append_decode(1, 1, 4, 1, 128, 256, [1], [n], 2, seed=n, chunk_cap=8192, tune={"decode_short_tokens": short})
+
+
+# head_dim 64 (half the row bytes, twice the pipeline stages, half the MMA steps)
+@pytest.mark.parametrize("n", [1, 17, 320, 321, 700])
+def test_head_dim_64_lengths(n):
+    run_append_decode(2, 1, 8, 2, 64, 256, [1, 0], [n], 3, seed=640 + n, D=64)
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(2, 2), (8, 2), (16, 1), (12, 4)])
+def test_head_dim_64_group_sizes(Hq, Hkv):
+    run_append_decode(2, 1, Hq, Hkv, 8, 24, [1, 0], [700], 4, seed=64 + Hq * 31 + Hkv, D=64)
+
+
+def test_head_dim_64_many_splits_ragged_batch_and_mixed_heads():
+    run_append_decode(2, 3, 8, 2, 16, 48, [1, 0], [9000, 37, 2600], 3, seed=641, chunk_cap=3000, D=64)
+    kvk = np.array([[1, 0], [0, 1]], dtype=np.uint8)
+    run_append_decode(2, 2, 8, 2, 16, 48, [0, 0], [5000, 300], 3, seed=642, kvk=kvk, chunk_cap=3000, D=64)
 
 
 def test_ragged_batch():
