@@ -21,7 +21,8 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All
  *     compute calls are asynchronous on that stream.  A handle is not thread-safe and
  *     calls on one handle must be issued in stream order on one stream at a time.
- *   - Tensors are bf16 (2-byte), row-major, innermost dimension head_dim = 128.
+ *   - Tensors are bf16 (2-byte), row-major, innermost dimension head_dim (128, or 64; the sizes
+ *     written as 128 below are head_dim).
  *     q/out of a call:   [tokens, n_q_heads, head_dim]
  *     k/v of a call:     [tokens, n_kv_heads, head_dim]
  *     `tokens` is the packed concatenation over the batch, sequence 0 first.
@@ -50,7 +51,8 @@ extern "C" {
 
 #define ZZ_OK 0
 #define ZZ_ERR_INVALID_ARG (-1) /* NULL pointer, index out of range, inconsistent sizes        */
-#define ZZ_ERR_UNSUPPORTED (-2) /* head_dim != 128, group size > 16, batch > ZZ_MAX_BATCH, ...  */
+#define ZZ_ERR_UNSUPPORTED (-2) /* head_dim not 64 or 128, group size > 16, batch > ZZ_MAX_BATCH,
+                                   FP8 or paged stores at head_dim 64, ...                      */
 #define ZZ_ERR_CAPACITY (-3)    /* len + n_new would exceed capacity[seq] of a retrieval store  */
 #define ZZ_ERR_WORKSPACE (-4)   /* arena or workspace smaller than zz_cache_query reported      */
 #define ZZ_ERR_CUDA (-5)        /* a CUDA runtime/driver call failed                            */
@@ -69,7 +71,7 @@ typedef struct zz_config {
     int32_t batch;                      /* sequences, 1 .. ZZ_MAX_BATCH                         */
     int32_t n_q_heads;
     int32_t n_kv_heads;                 /* divides n_q_heads; group size <= 16                  */
-    int32_t head_dim;                   /* must be 128                                          */
+    int32_t head_dim;                   /* 128 or 64 (FP8 and paged stores: 128 only)           */
     int32_t sink;                       /* S >= 0                                               */
     int32_t recent;                     /* W >= 1                                               */
     int32_t max_new_tokens;             /* largest sum of n_new over the batch in one prefill

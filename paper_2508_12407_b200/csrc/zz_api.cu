@@ -587,7 +587,6 @@ int launch_prefill_group(zz_cache* c, int layer, int kind, const CUtensorMap* tq
     const int nR = c->nR[layer];
     const int Hg = (kind == ZZ_KIND_RETRIEVAL) ? nR : c->Hkv - nR;
     if (Hg == 0) return ZZ_OK;
-    if (c->D != kD) return ZZ_ERR_UNSUPPORTED;   // TEMP: prefill at head_dim 64
     const bool fp8 = c->fp8 && kind == ZZ_KIND_RETRIEVAL;
     if (fp8) {
         // rows already stored are expanded to bf16 in the scratch (exactly: an FP8 value is a bf16

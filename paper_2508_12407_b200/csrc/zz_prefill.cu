@@ -33,7 +33,7 @@ namespace {
 
 constexpr int kTile = 128;
 constexpr int kSubBytes = 128 * 128;        // [128 rows][64 bf16] sub-tile, 128-byte swizzled
-constexpr int kTileBytes = 2 * kSubBytes;   // a full [128][128] bf16 tile
+constexpr int kTileBytes = 2 * kSubBytes;   // a full [128][128] bf16 tile (head_dim 128; half of it at head_dim 64)
 constexpr int kStages = 4;                  // K/V tiles held at once: two pair slots of (V_j, K_{j+1})
 constexpr int kPairs = 2;                   // one full / empty barrier per pair: what an iteration uses, it uses together
 constexpr int kThreads = 384;                // three warpgroups: softmax tile 0, softmax tile 1, TMA + MMA
@@ -54,7 +54,10 @@ constexpr int kPolyEvery = ZZ_POLY_EVERY;   // one pair in kPolyEvery takes the 
 
 // instruction descriptor: fp32 accumulate, bf16 A and B, M = 128, N = 128
 constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);   // B (= V) is MN-major
+// P V: N = head_dim, B (= V) is MN-major
+__host__ __device__ constexpr uint32_t idesc_pv(int hd) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)hd >> 3) << 17) | ((128u >> 4) << 24);
+}
 
 struct Shared {
     uint64_t q_full;
@@ -384,7 +387,9 @@ __device__ __forceinline__ int item_key(const PrefillParams& p, int idx) {
 // the item loops below then run once and every running counter folds to a constant.  Persistent
 // CTAs gain ~10 % on the short items of streaming layers and 2-5 % on retrieval chunks of 2K-8K
 // tokens; on 32K chunks the two time the same.
-template <bool kPersistent>
+// HD = head_dim: 128, or 64 (Q, K and V tiles are then one 64-column sub-tile, Q K^T has four MMA steps
+// instead of eight, P V has N = 64, and O takes 64 columns of tensor memory).
+template <bool kPersistent, int HD>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q,
                const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
@@ -393,6 +398,8 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
     __shared__ Shared sh;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sm_q = smem_base;                       // two Q tiles
+    constexpr int kTileB = (HD / 64) * kSubBytes;          // bytes of a Q, K or V tile
+    constexpr uint32_t kIdescPV = idesc_pv(HD);
     const uint32_t sm_kv = smem_base + 2 * kTileBytes;     // kStages K/V tiles
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -506,18 +513,18 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                 // paged retrieval store: a store tile is one page (tiles and pages are both 128 tokens)
                 const bool paged = p.page_table != nullptr && p.kind == ZZ_KIND_RETRIEVAL;
                 const int* const tbl = paged ? p.page_table + sd.tbl + it.hg : nullptr;
-                const int k_row0 = (int)(sd.k_off[p.kind] / kD + (paged ? 0ll : (long long)it.hg * slots_per_head));
-                const int v_row0 = (int)(sd.v_off[p.kind] / kD + (paged ? 0ll : (long long)it.hg * slots_per_head));
+                const int k_row0 = (int)(sd.k_off[p.kind] / HD + (paged ? 0ll : (long long)it.hg * slots_per_head));
+                const int v_row0 = (int)(sd.v_off[p.kind] / HD + (paged ? 0ll : (long long)it.hg * slots_per_head));
                 const int src_head = p.head_list[p.kv_head0 + it.hg];
                 const int tok0 = p.tok_off[it.b];
                 const int qh = p.q_head0 + it.hg * p.G + it.g0;
                 if (k > 0) mbar_wait(&sh.q_empty, (k - 1) & 1, &sh, p.status);
-                mbar_expect_tx(&sh.q_full, it.active1 ? 2 * kTileBytes : kTileBytes);
+                mbar_expect_tx(&sh.q_full, it.active1 ? 2 * kTileB : kTileB);
                 tma_load_3d(sm_q, &tmap_q, 0, qh, tok0 + it.r0, &sh.q_full);
-                tma_load_3d(sm_q + kSubBytes, &tmap_q, 64, qh, tok0 + it.r0, &sh.q_full);
+                if (HD == 128) tma_load_3d(sm_q + kSubBytes, &tmap_q, 64, qh, tok0 + it.r0, &sh.q_full);
                 if (it.active1) {
-                    tma_load_3d(sm_q + kTileBytes, &tmap_q, 0, qh + 1, tok0 + it.r0, &sh.q_full);
-                    tma_load_3d(sm_q + kTileBytes + kSubBytes, &tmap_q, 64, qh + 1, tok0 + it.r0, &sh.q_full);
+                    tma_load_3d(sm_q + kTileB, &tmap_q, 0, qh + 1, tok0 + it.r0, &sh.q_full);
+                    if (HD == 128) tma_load_3d(sm_q + kTileB + kSubBytes, &tmap_q, 64, qh + 1, tok0 + it.r0, &sh.q_full);
                 }
                 // pair pi of the item: pi = 0 holds K_0 alone, pi = j + 1 holds (V_j, K_{j+1}), the last one
                 // V_{n-1} alone; slot = running pair count % 2, V in the slot's first tile, K in its second
@@ -525,23 +532,23 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                     const int slot = u_glob % kPairs;
                     mbar_wait(&sh.kv_empty[slot], ((u_glob / kPairs) & 1) ^ 1, &sh, p.status);
                     const bool has_v = pi > 0, has_k = pi < it.n_tiles;
-                    mbar_expect_tx(&sh.kv_full[slot], (has_v && has_k) ? 2 * kTileBytes : kTileBytes);
+                    mbar_expect_tx(&sh.kv_full[slot], (has_v && has_k) ? 2 * kTileB : kTileB);
 #pragma unroll
                     for (int is_k = 0; is_k < 2; ++is_k) {
                         if (is_k ? !has_k : !has_v) continue;
                         bool is_chunk;
                         int start;
                         plan_tile(it.plan, is_k ? pi : pi - 1, is_chunk, start);
-                        const uint32_t dst = sm_kv + (slot * 2 + is_k) * kTileBytes;
+                        const uint32_t dst = sm_kv + (slot * 2 + is_k) * kTileB;
                         if (is_chunk) {
                             const CUtensorMap* m = is_k ? &tmap_k : &tmap_v;
                             tma_load_3d(dst, m, 0, src_head, tok0 + start, &sh.kv_full[slot]);
-                            tma_load_3d(dst + kSubBytes, m, 64, src_head, tok0 + start, &sh.kv_full[slot]);
+                            if (HD == 128) tma_load_3d(dst + kSubBytes, m, 64, src_head, tok0 + start, &sh.kv_full[slot]);
                         } else {
                             const int row = (is_k ? k_row0 : v_row0) +
                                             (paged ? tbl[(start >> 7) * p.Hg] * (int)(kPageElems / kD) : start);
                             tma_load_2d(dst, &tmap_arena, 0, row, &sh.kv_full[slot]);
-                            tma_load_2d(dst + kSubBytes, &tmap_arena, 64, row, &sh.kv_full[slot]);
+                            if (HD == 128) tma_load_2d(dst + kSubBytes, &tmap_arena, 64, row, &sh.kv_full[slot]);
                         }
                     }
                 }
@@ -563,7 +570,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
             const uint64_t dv = make_desc(sm_kv, kSubBytes, 1024);  // V tile of pair slot 0, MN-major
             const uint32_t dq_lo = (uint32_t)dq, dk_lo = (uint32_t)dk, dv_lo = (uint32_t)dv;
             const uint32_t dkm_hi = (uint32_t)(dq >> 32), dv_hi = (uint32_t)(dv >> 32);
-            constexpr uint32_t kTile16 = kTileBytes >> 4;
+            constexpr uint32_t kTile16 = kTileB >> 4;
             // Counters that run across the items of this CTA (barrier phases never restart):
             uint32_t u_glob = 0;          // K/V pairs consumed
             uint32_t ph[2] = {0, 0};      // S/P tiles handled per query tile (tile 1 only in items that have it)
@@ -582,7 +589,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                     // S_t = Q_t K_0^T
                     for (int t = 0; t < n_act; ++t) {
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
+                        for (int kk = 0; kk < HD / 16; ++kk) {
                             const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
                             mma_ss(tmem_u + t * 256, dq_lo + t * kTile16 + off16,
                                    dk_lo + ((u_glob % kPairs) * 2 + 1) * kTile16 + off16, dkm_hi, dkm_hi, kIdescQK, kk > 0);
@@ -615,7 +622,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                                        (kk > 0) || (j > 0));
                             // S_t = Q_t K_{j+1}^T (not after the last tile)
 #pragma unroll
-                            for (int kk = 0; kk < 8; ++kk) {
+                            for (int kk = 0; kk < HD / 16; ++kk) {
                                 const uint32_t off16 = (kk >> 2) * (kSubBytes >> 4) + (kk & 3) * 2;
                                 mma_ss_if(more, t_st, dqt + off16, dkj + off16, dkm_hi, dkm_hi, kIdescQK, kk > 0);
                             }
@@ -832,7 +839,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                         // PV of the previous tile has completed (its commit precedes s_full), so O is stable
                         float o[32];
 #pragma unroll 1
-                        for (int c = 0; c < 4; ++c) {
+                        for (int c = 0; c < HD / 32; ++c) {
                             tmem_ld32(t_o + c * 32, o);
                             tmem_wait_ld();
 #pragma unroll
@@ -856,14 +863,17 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
             // XOR-swizzled by row) and writes them out with every 256-byte row covered by 16
             // consecutive lanes, instead of one lane per row.  (The Q buffers are not used for this:
             // the producer may already be loading the next item's Q.)
+            // (at head_dim 64 a row is 128 bytes: 8 pieces, 8 lanes per row)
+            constexpr int kPieces = HD / 8;                    // 16-byte pieces of an output row
+            constexpr int kRowB = HD * 2;
             const uint32_t stage = sm_epi + (uint32_t)(warp * 4096);
-            const int piece_r = lane & 15, half_r = lane >> 4;
+            const int piece_r = lane % kPieces, half_r = lane / kPieces;
             const long long row0 = (long long)p.tok_off[b] + r0 + quarter * 32;
-            __nv_bfloat16* obase = p.out + (long long)(p.q_head0 + hg * p.G + g0 + t) * kD + piece_r * 8;
+            __nv_bfloat16* obase = p.out + (long long)(p.q_head0 + hg * p.G + g0 + t) * HD + piece_r * 8;
 #pragma unroll 1
             for (int h = 0; h < 2; ++h) {
 #pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < HD / 32; ++c) {
                     float o[32];
                     tmem_ld32(t_o + c * 32, o);
                     tmem_wait_ld();
@@ -876,19 +886,19 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                             const uint32_t w3 = pack_bf16(o[8 * i + 6] * inv, o[8 * i + 7] * inv);
                             const uint32_t piece = (uint32_t)(c * 4 + i);
                             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                                         ::"r"(stage + (lane & 15) * 256 + ((piece ^ (lane & 15)) << 4)),
+                                         ::"r"(stage + (lane & 15) * kRowB + ((piece ^ (lane & (kPieces - 1))) << 4)),
                                            "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
                         }
                     }
                 }
                 __syncwarp();
 #pragma unroll 4
-                for (int i = 0; i < 8; ++i) {
-                    const int sr = 2 * i + half_r;                         // row inside the staged 16
+                for (int i = 0; i < kPieces / 2; ++i) {
+                    const int sr = (32 / kPieces) * i + half_r;            // row inside the staged 16
                     const int lr = 16 * h + sr;                            // row inside the warp's 32
                     uint32_t w0, w1, w2, w3;
                     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
-                                 : "r"(stage + sr * 256 + ((piece_r ^ sr) << 4)) : "memory");
+                                 : "r"(stage + sr * kRowB + ((piece_r ^ (sr & (kPieces - 1))) << 4)) : "memory");
                     if (r0 + quarter * 32 + lr < C)
                         *reinterpret_cast<uint4*>(obase + (row0 + lr) * p.tok_stride) = make_uint4(w0, w1, w2, w3);
                 }
@@ -939,26 +949,35 @@ cudaError_t prefill_setup() {
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(prefill_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(prefill_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(prefill_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(prefill_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(prefill_kernel<false, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    return e;
+}
+
+template <bool kPersistent, int HD>
+static void launch_one(int grid, const PrefillParams& pp, const void* tq, const void* tk, const void* tv, const void* ta,
+                       cudaStream_t s) {
+    prefill_kernel<kPersistent, HD><<<grid, kThreads, kSmemBytes, s>>>(pp, *static_cast<const CUtensorMap*>(tq),
+                                                                     *static_cast<const CUtensorMap*>(tk),
+                                                                     *static_cast<const CUtensorMap*>(tv),
+                                                                     *static_cast<const CUtensorMap*>(ta));
 }
 
 cudaError_t launch_prefill(const PrefillParams& p, const void* tq, const void* tk, const void* tv,
                            const void* ta, int n_items, cudaStream_t s) {
     PrefillParams pp = p;
     pp.n_items = n_items;
-    if (g_num_sms > 0 && n_items > g_num_sms) {
-        // persistent CTAs, one per SM (tensor memory and shared memory allow no more)
-        prefill_kernel<true><<<g_num_sms, kThreads, kSmemBytes, s>>>(pp, *static_cast<const CUtensorMap*>(tq),
-                                                                   *static_cast<const CUtensorMap*>(tk),
-                                                                   *static_cast<const CUtensorMap*>(tv),
-                                                                   *static_cast<const CUtensorMap*>(ta));
+    if (p.D != 128 && p.D != 64) return cudaErrorInvalidValue;
+    // persistent CTAs, one per SM (tensor memory and shared memory allow no more), when there are more items than SMs
+    const bool persistent = g_num_sms > 0 && n_items > g_num_sms;
+    if (p.D == 128) {
+        if (persistent) launch_one<true, 128>(g_num_sms, pp, tq, tk, tv, ta, s);
+        else launch_one<false, 128>(n_items, pp, tq, tk, tv, ta, s);
     } else {
-        prefill_kernel<false><<<n_items, kThreads, kSmemBytes, s>>>(pp, *static_cast<const CUtensorMap*>(tq),
-                                                                  *static_cast<const CUtensorMap*>(tk),
-                                                                  *static_cast<const CUtensorMap*>(tv),
-                                                                  *static_cast<const CUtensorMap*>(ta));
+        if (persistent) launch_one<true, 64>(g_num_sms, pp, tq, tk, tv, ta, s);
+        else launch_one<false, 64>(n_items, pp, tq, tk, tv, ta, s);
     }
     count_launch();
     return cudaGetLastError();

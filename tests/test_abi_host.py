@@ -49,7 +49,7 @@ def make_cfg(**kw):
     cap = np.array(kw.get("cap", [1024] * B), dtype=np.int32)
     cfg = binding.ZZConfig(L, B, kw.get("Hq", 8), kw.get("Hkv", 2), kw.get("D", 128), kw.get("S", 64),
                            kw.get("W", 256), kw.get("max_new", 2048), kw.get("scale", 0.088),
-                           kinds.ctypes.data, None, cap.ctypes.data)
+                           kinds.ctypes.data, None, cap.ctypes.data, kw.get("fp8", 0))
     cfg._keep = (kinds, cap)
     return cfg
 
@@ -70,7 +70,10 @@ def test_query_sizes(lib):
 
 
 @pytest.mark.parametrize("kw,code", [
-    (dict(D=64), binding.ZZ_ERR_UNSUPPORTED),
+    (dict(D=96), binding.ZZ_ERR_UNSUPPORTED),
+    (dict(D=256), binding.ZZ_ERR_UNSUPPORTED),
+    (dict(D=64, fp8=1), binding.ZZ_ERR_UNSUPPORTED),
+    (dict(fp8=2), binding.ZZ_ERR_INVALID_ARG),
     (dict(Hq=6, Hkv=4), binding.ZZ_ERR_UNSUPPORTED),
     (dict(Hq=34, Hkv=2), binding.ZZ_ERR_UNSUPPORTED),
     (dict(B=65, cap=[8] * 65, max_new=100), binding.ZZ_ERR_UNSUPPORTED),
@@ -83,6 +86,25 @@ def test_query_sizes(lib):
 def test_query_rejects_bad_configs(lib, kw, code):
     rc, _, _ = query(lib, make_cfg(**kw))
     assert rc == code
+
+
+def test_query_sizes_head_dim_64_fp8_and_paged(lib):
+    rc, a, w = query(lib, make_cfg(D=64))
+    assert rc == 0
+    expect = 2 * (2 * 1024 * 128) + 2 * (2 * 320 * 128)        # rows of 64 bf16
+    assert expect <= a <= expect + 128 * 128 + 256
+    # FP8 retrieval stores: 128 code bytes + 1 scale byte per row, then one layer's worth of bf16 scratch
+    rc, a8, _ = query(lib, make_cfg(fp8=1))
+    assert rc == 0
+    codes = 2 * (2 * 1024 * 128) + 2 * (2 * 1024)
+    ring = 2 * (2 * 320 * 256)
+    scratch = 2 * (2 * 1024 * 256)
+    assert codes + ring + scratch <= a8 <= codes + ring + scratch + 4 * 256 + 128 * 256 + 256
+    a2, w2 = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    cfg = make_cfg(D=64)
+    assert lib.zz_cache_query_paged(ctypes.byref(cfg), 8, ctypes.byref(a2), ctypes.byref(w2)) == binding.ZZ_ERR_UNSUPPORTED
+    cfg = make_cfg(fp8=1)
+    assert lib.zz_cache_query_paged(ctypes.byref(cfg), 8, ctypes.byref(a2), ctypes.byref(w2)) == binding.ZZ_ERR_UNSUPPORTED
 
 
 def test_null_arguments(lib):

@@ -16,16 +16,15 @@ def _built():
 
 
 def run_prefill(L, B, Hq, Hkv, S, W, kinds, chunk_plans, seed, kvk=None, n_decode=0, sample_rows=None,
-                pool_pages=0):
+                pool_pages=0, D=128):
     """chunk_plans[b] = list of chunk sizes of sequence b (a 0 skips the sequence in that call)."""
-    D = 128
     scale = 1.0 / np.sqrt(D)
     total = [int(sum(pl)) for pl in chunk_plans]
     cap = [t + n_decode + 1 for t in total]
     max_new = max(sum(pl[r] if r < len(pl) else 0 for pl in chunk_plans)
                   for r in range(max(len(pl) for pl in chunk_plans)))
     cache = binding.ZigzagCache(L, B, Hq, Hkv, S, W, kinds, cap, max(max_new, B), kvhead_is_retrieval=kvk,
-                                pool_pages=pool_pages)
+                                pool_pages=pool_pages, head_dim=D)
     w = inputs.Workload("t", L, B, Hq, Hkv, D, S, W, int(sum(kinds)), 0, 0, n_decode, seed=seed)
 
     def kv_kinds(l):
@@ -198,3 +197,23 @@ def test_scores_of_very_different_magnitude():
         assert_close(to_bits(out), o.rows(q, [2 * C], scale=scale), f"layer {l} decode")
     assert cache.last_status() == 0
     cache.close()
+
+
+# head_dim 64: tiles of one 64-column sub-tile, four MMA steps per Q K^T, N = 64 for P V
+def test_head_dim_64_single_shot_and_chunked():
+    run_prefill(2, 1, 8, 2, 64, 256, [1, 0], [[2048]], seed=6401, n_decode=2, D=64)
+    run_prefill(2, 1, 8, 2, 16, 48, [1, 0], [[300, 77, 1, 500, 129]], seed=6402, n_decode=2, D=64)
+
+
+def test_head_dim_64_ragged_batch_odd_heads_and_mixed_layer():
+    run_prefill(2, 3, 6, 2, 16, 48, [1, 0], [[700, 50], [33, 0], [128, 300]], seed=6403, n_decode=1, D=64)
+    kvk = np.array([[1, 0], [0, 1]], dtype=np.uint8)
+    run_prefill(2, 2, 8, 2, 16, 48, [0, 0], [[400, 300], [129, 64]], seed=6404, kvk=kvk, n_decode=1, D=64)
+
+
+def test_head_dim_64_many_items_persistent_launch():
+    # more work items than SMs, so the persistent instantiation and the per-CTA item order run
+    run_prefill(1, 1, 32, 8, 16, 48, [1], [[4096]], seed=6405, D=64,
+                sample_rows=lambda P, c: [0, 1, 127, 128, 129, 1000, 2047, 2048, 4095])
+    run_prefill(1, 1, 32, 8, 128, 256, [0], [[4096, 2048]], seed=6406, D=64,
+                sample_rows=lambda P, c: [0, 1, 127, 128, 383, 384, 385, 1000, c - 1])
