@@ -56,7 +56,7 @@ using zz::SeqDesc;
 namespace {
 
 constexpr int kMaxSplits = zz::kDecodeMaxSplits;   // the decode kernel keeps per-split factors in 128-entry rows
-constexpr int kMaxSlots = 512;    // upper bound of CTAs a long-store decode plan may use (2 per SM)
+constexpr int kMaxSlots = 512;    // upper bound of CTAs a long-store decode plan may use (2 or 3 per SM)
 constexpr size_t kAlign = 256;
 
 size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
@@ -481,7 +481,7 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
         n[b] = (kind == ZZ_KIND_RETRIEVAL) ? len : (len < c->ring ? len : c->ring);
     }
     int warps = 4;
-    // (the FP8 kernel's 4-warp CTAs fit three to an SM, the bf16 kernel's two)
+    // (the FP8 kernels' 4-warp CTAs fit three to an SM, the bf16 kernel's two)
     plan_splits(c, n, Hg, &warps, p.chunk, p.split_start, d_layer_ids ? n_multi : 1, fp8 ? 3 : 2);
     const int items = p.split_start[c->B] * Hg;
     const int pk = (kind == ZZ_KIND_RETRIEVAL) ? zz::kProfDecodeR : zz::kProfDecodeS;

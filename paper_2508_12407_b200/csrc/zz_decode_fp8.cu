@@ -14,6 +14,8 @@
 //   * the V scale of each token multiplies its probability before that is rounded to f16, relative to
 //     the largest V scale the warp has met so far (the accumulators are rescaled when it grows), so the
 //     f16 operand never overflows and rows with tiny scales simply contribute little.
+// Groups of up to eight query heads run decode_fp8t_kernel, which computes both products transposed
+// (see there); larger groups run decode_fp8_kernel.
 // An 8-bit row is 128 bytes: ldmatrix moves it as 16-bit units, which puts four consecutive dims of a
 // token into a thread's register for K (the query fragments are loaded in the matching order) and two
 // dims of two consecutive tokens for V (a byte permute separates them; an accumulator tile therefore
@@ -454,6 +456,271 @@ __global__ void __launch_bounds__(kWarps * 32, 12 / kWarps) decode_fp8_kernel(co
                                      p.appended && p.bump_len, len_p, out_p, part_o_p, part_ml_p, counters_p, seq_counters_p);
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// The same decode step with the products transposed, for groups of up to eight query heads.
+//   S^T = K Q^T:  tokens are the 16 rows of the MMA tile, the group's query heads its 8 columns;
+//   O^T = V^T P^T: 16 head dims are the rows, the query heads the columns, the block's 16 tokens the
+//   contraction.
+// A 16 x 8 tile wastes nothing on a group of eight (or four) heads, where the untransposed kernel
+// fills at most half of its 16 query rows: half the MMAs, half the accumulator registers (32), half
+// the query registers, and with them room for more warps per SM, which is what this issue-bound kernel
+// needs.  The probabilities come out of the first product with tokens along the rows and are needed
+// with tokens along the contraction: one movmatrix per 8 x 8 block transposes them.
+// Thread (grp, tig) of a warp holds, per 16-token block: scores of tokens grp and grp + 8 for heads
+// 2 tig and 2 tig + 1; its accumulator tile c holds dims 16 c + 2 grp (+ 1) of those two heads.
+// ---------------------------------------------------------------------------------------------
+constexpr int kStagesT = 4;
+constexpr int kWarpSmemT = kStagesT * kStageF8;   // 16896 B per warp: 4 warps 66 KiB (three CTAs per SM; four CTAs of
+                                                  // three stages at 128 registers timed the same and spilled in the merge)
+
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+    uint32_t r;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(r) : "r"(x));
+    return r;
+}
+
+template <int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 12 / kWarps) decode_fp8t_kernel(const DecodeParams p) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    __shared__ int s_is_last;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int grp = lane >> 2, tig = lane & 3;
+
+    if (p.gdc_wait == 2) asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    const int li = p.layer_ids ? p.layer_ids[blockIdx.y] : 0;
+    int* const len_p = p.len + (long long)li * p.st_len;
+    const __nv_bfloat16* const q_p = p.q + (long long)li * p.st_q;
+    __nv_bfloat16* const out_p = p.out + (long long)li * p.st_q;
+    unsigned int* const counters_p = p.counters + (long long)li * p.st_cnt;
+    unsigned int* const seq_counters_p = p.seq_counters + (long long)li * p.st_cnt;
+    float* const part_o_p = p.part_o + (long long)li * p.st_part * kD;
+    float* const part_ml_p = p.part_ml + (long long)li * p.st_part * 2;
+
+    const int item = blockIdx.x;
+    int b = 0;
+    while (b + 1 < p.B && item >= p.split_start[b + 1] * p.Hg) ++b;
+    const int local = item - p.split_start[b] * p.Hg;
+    const int hg = local % p.Hg;
+    const int split = local / p.Hg;
+    const int nsplit = p.split_start[b + 1] - p.split_start[b];
+    if (nsplit > p.max_splits || p.max_splits > kDecodeMaxSplits) {
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, ZZ_ERR_UNSUPPORTED);
+        return;
+    }
+    const int len_old = len_p[b];
+    const SeqDesc sd = p.layer_ids ? p.desc_table[(long long)li * p.B + b] : p.sd[b];
+    if (p.appended && len_old >= sd.cap) {
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, ZZ_ERR_CAPACITY);
+        return;
+    }
+    const int n = len_old + (p.appended ? 1 : 0);
+    const int cap16 = fp8_cap16(sd.cap);
+    const unsigned char* const arena8 = reinterpret_cast<const unsigned char*>(p.arena);
+    const unsigned char* const kc = arena8 + 2 * sd.k_off[ZZ_KIND_RETRIEVAL] + (long long)hg * sd.cap * kD;
+    const unsigned char* const vc = arena8 + 2 * sd.v_off[ZZ_KIND_RETRIEVAL] + (long long)hg * sd.cap * kD;
+    const unsigned char* const ks = arena8 + fp8_kscale_byte_off(sd.v_off[ZZ_KIND_RETRIEVAL], p.Hg, sd.cap) + (long long)hg * cap16;
+    const unsigned char* const vs = ks + (long long)p.Hg * cap16;
+
+    const int s0 = min(split * p.chunk[b], n);
+    const int s1 = (split == nsplit - 1) ? n : min(n, s0 + p.chunk[b]);
+    const int nblk = (s1 - s0 + kBlk - 1) / kBlk;
+    const int my_blocks = (nblk > warp) ? (nblk - warp + kWarps - 1) / kWarps : 0;
+
+    // ---- query fragments (B operand of S^T = K Q^T): head grp, dims 16 kk + 4 tig + {0, 1} and + {2, 3},
+    // each row scaled by a power of two into f16's range ----------------------------------------------
+    const int G = p.G;
+    const __nv_bfloat16* qb = q_p + ((long long)b * p.q_tok_stride) + (long long)(p.q_head0 + hg * G) * kD;
+    uint32_t qf[8][2];
+    float qmul[2];
+    {
+        uint2 raw[8];
+        uint32_t amax = 0;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+            raw[kk] = (grp < G) ? *reinterpret_cast<const uint2*>(qb + grp * kD + kk * 16 + tig * 4) : make_uint2(0u, 0u);
+            amax = max(max(amax, raw[kk].x & 0x7FFFu), max((raw[kk].x >> 16) & 0x7FFFu, max(raw[kk].y & 0x7FFFu, (raw[kk].y >> 16) & 0x7FFFu)));
+        }
+        amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+        amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+        int kq = (int)(amax >> 7);
+        kq = kq > 253 ? 253 : kq;
+        const float down = pow2_of_byte(254 - kq);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+            qf[kk][0] = pack_f16(__uint_as_float(raw[kk].x << 16) * down, __uint_as_float(raw[kk].x & 0xFFFF0000u) * down);
+            qf[kk][1] = pack_f16(__uint_as_float(raw[kk].y << 16) * down, __uint_as_float(raw[kk].y & 0xFFFF0000u) * down);
+        }
+        // this thread's score columns are heads 2 tig and 2 tig + 1: their factors live in the lanes of those rows
+        const float mine = p.scale_log2 * pow2_of_byte(kq);
+        qmul[0] = __shfl_sync(0xffffffffu, mine, (2 * tig) * 4);
+        qmul[1] = __shfl_sync(0xffffffffu, mine, (2 * tig + 1) * 4);
+    }
+
+    float o[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+    float m_run[2] = {-INFINITY, -INFINITY};
+    float l_run[2] = {0.f, 0.f};                      // partial: this thread's two tokens of every block
+    int eref = 0;
+
+    const uint32_t wbase = smem_u32(smem) + warp * kWarpSmemT;
+    uint64_t l2_policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(l2_policy));
+
+#pragma unroll
+    for (int s = 0; s < kStagesT - 1; ++s) {
+        if (s < my_blocks) {
+            const int tok0 = s0 + (warp + s * kWarps) * kBlk;
+            load_block_fp8(wbase + s * kStageF8, kc, vc, ks, vs, tok0, s1, lane, l2_policy);
+        }
+        cp_async_commit();
+    }
+
+    for (int it = 0; it < my_blocks; ++it) {
+        {
+            const int nx = it + kStagesT - 1;
+            if (nx < my_blocks) {
+                const int tok0 = s0 + (warp + nx * kWarps) * kBlk;
+                load_block_fp8(wbase + (nx % kStagesT) * kStageF8, kc, vc, ks, vs, tok0, s1, lane, l2_policy);
+            }
+            cp_async_commit();
+        }
+        cp_async_wait<kStagesT - 1>();
+        __syncwarp();
+
+        const uint32_t sk = wbase + (it % kStagesT) * kStageF8;
+        const uint32_t sv = sk + kCodeBytes;
+        const int tok0 = s0 + (warp + it * kWarps) * kBlk;
+        const int valid = s1 - tok0;   // >= 1
+
+        // scale bytes of this thread's two tokens, grp and grp + 8
+        uint32_t kb0, kb1, vb0, vb1;
+        asm volatile("ld.shared.u8 %0, [%1];" : "=r"(kb0) : "r"(sk + 2 * kCodeBytes + grp));
+        asm volatile("ld.shared.u8 %0, [%1];" : "=r"(kb1) : "r"(sk + 2 * kCodeBytes + 8 + grp));
+        asm volatile("ld.shared.u8 %0, [%1];" : "=r"(vb0) : "r"(sk + 2 * kCodeBytes + 16 + grp));
+        asm volatile("ld.shared.u8 %0, [%1];" : "=r"(vb1) : "r"(sk + 2 * kCodeBytes + 24 + grp));
+        const bool ok0 = grp < valid, ok1 = grp + 8 < valid;
+        if (!ok0) { kb0 = 0; vb0 = 0; }
+        if (!ok1) { kb1 = 0; vb1 = 0; }
+
+        // S^T = K Q^T
+        float sc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int pc = 0; pc < 4; ++pc) {
+            const int r = (lane & 7) + (((lane >> 3) & 1) << 3);
+            const int c = pc * 2 + (lane >> 4);
+            uint32_t m0, m1, m2, m3, a0, a1, a2, a3;
+            ldmatrix_x4(sk + r * kD + ((c ^ (r & 7)) << 4), m0, m1, m2, m3);
+            e4m3x4_to_f16x2x2(m0, a0, a2);      // token grp:     dims 4 tig + {0, 1} | {2, 3} of piece 2 pc
+            e4m3x4_to_f16x2x2(m1, a1, a3);      // token grp + 8
+            mma_f16(sc, a0, a1, a2, a3, qf[2 * pc][0], qf[2 * pc][1]);
+            e4m3x4_to_f16x2x2(m2, a0, a2);      // piece 2 pc + 1
+            e4m3x4_to_f16x2x2(m3, a1, a3);
+            mma_f16(sc, a0, a1, a2, a3, qf[2 * pc + 1][0], qf[2 * pc + 1][1]);
+        }
+
+        // the block's largest V scale (all lanes: 16 tokens spread over the 8 row groups)
+        int vmax = max((int)vb0, (int)vb1);
+        vmax = max(vmax, __shfl_xor_sync(0xffffffffu, vmax, 4));
+        vmax = max(vmax, __shfl_xor_sync(0xffffffffu, vmax, 8));
+        vmax = max(vmax, __shfl_xor_sync(0xffffffffu, vmax, 16));
+        if (vmax > eref) {
+            const float f = pow2_of_byte(max(eref - vmax + 127, 0));
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { o[i][0] *= f; o[i][1] *= f; o[i][2] *= f; o[i][3] *= f; }
+            eref = vmax;
+        }
+        const float vf0 = pow2_of_byte(max((int)vb0 - eref + 127, 0)), vf1 = pow2_of_byte(max((int)vb1 - eref + 127, 0));
+        const float kf0 = pow2_of_byte((int)kb0), kf1 = pow2_of_byte((int)kb1);
+
+        float pr[4];                                  // probabilities: [token grp | grp + 8][head 2 tig | 2 tig + 1]
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            float t0 = ok0 ? sc[e] * (qmul[e] * kf0) : -INFINITY;
+            float t1 = ok1 ? sc[2 + e] * (qmul[e] * kf1) : -INFINITY;
+            float mx = fmaxf(t0, t1);
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+            const float m_new = fmaxf(m_run[e], mx);        // finite: token 0 of a block is always valid
+            t0 = fast_exp2(t0 - m_new);
+            t1 = fast_exp2(t1 - m_new);
+            if (__any_sync(0xffffffffu, m_new > m_run[e])) {
+                const float alpha = fast_exp2(m_run[e] - m_new);   // 0 on the first block
+                l_run[e] = l_run[e] * alpha + (t0 + t1);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    o[i][e] *= alpha;
+                    o[i][2 + e] *= alpha;
+                }
+            } else {
+                l_run[e] += t0 + t1;
+            }
+            m_run[e] = m_new;
+            pr[e] = t0 * vf0;
+            pr[2 + e] = t1 * vf1;
+        }
+        // P^T for the second product: tokens along the contraction, heads along the columns
+        const uint32_t pb0 = movmatrix_trans(pack_f16(pr[0], pr[1]));   // tokens 2 tig, 2 tig + 1 of head grp
+        const uint32_t pb1 = movmatrix_trans(pack_f16(pr[2], pr[3]));   // tokens 8 + 2 tig, 9 + 2 tig
+
+        // O^T += V^T P^T: a transposed 16-bit unit holds dims (2 grp, 2 grp + 1) of tokens 2 tig (low half)
+        // and 2 tig + 1; the permute puts the two tokens of each dim side by side: rows grp and grp + 8 of the
+        // MMA tile are dims 2 grp and 2 grp + 1 of the piece
+#pragma unroll
+        for (int pc = 0; pc < 4; ++pc) {
+            const int r = (lane & 7) + (((lane >> 3) & 1) << 3);
+            const int c = pc * 2 + (lane >> 4);
+            uint32_t m0, m1, m2, m3, a0, a1, a2, a3;
+            ldmatrix_x4_trans(sv + r * kD + ((c ^ (r & 7)) << 4), m0, m1, m2, m3);
+            e4m3x4_to_f16x2x2(__byte_perm(m0, 0u, 0x3120), a0, a1);     // tokens 2 tig, + 1:   dim 2 grp | 2 grp + 1
+            e4m3x4_to_f16x2x2(__byte_perm(m1, 0u, 0x3120), a2, a3);     // tokens 8 + 2 tig, + 1
+            mma_f16(o[2 * pc], a0, a1, a2, a3, pb0, pb1);
+            e4m3x4_to_f16x2x2(__byte_perm(m2, 0u, 0x3120), a0, a1);
+            e4m3x4_to_f16x2x2(__byte_perm(m3, 0u, 0x3120), a2, a3);
+            mma_f16(o[2 * pc + 1], a0, a1, a2, a3, pb0, pb1);
+        }
+        __syncwarp();
+    }
+    cp_async_wait<0>();
+    if (p.gdc_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    // ---- stage the warp's results: rows = query heads, fp32 -------------------------------------------
+    {
+        const float f = pow2_of_byte(eref);
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 4);
+            l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 8);
+            l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 16);
+        }
+        __syncthreads();   // every warp is done with its pipeline memory
+        float* sm_o = reinterpret_cast<float*>(smem);                  // [kWarps][16][128]
+        float* sm_ml = sm_o + kWarps * 16 * kD;                        // [kWarps][16][2]
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int head = 2 * tig + e;
+            if (head < G) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    *reinterpret_cast<float2*>(sm_o + (warp * 16 + head) * kD + 16 * i + 2 * grp) =
+                        make_float2(o[i][e] * f, o[i][2 + e] * f);
+                if (grp == 0) {
+                    sm_ml[(warp * 16 + head) * 2 + 0] = m_run[e];
+                    sm_ml[(warp * 16 + head) * 2 + 1] = l_run[e];
+                }
+            }
+        }
+        __syncthreads();
+    }
+    finish_item_tail<kWarps, kD>(p, smem, &s_is_last, item, b, hg, nsplit, len_old, p.appended && p.bump_len, len_p, out_p,
+                                 part_o_p, part_ml_p, counters_p, seq_counters_p);
+}
+
 template <bool HI, int kWarps>
 cudaError_t setup_one_fp8() {
     return cudaFuncSetAttribute(decode_fp8_kernel<HI, kWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -467,6 +734,10 @@ cudaError_t decode_fp8_setup() {
     if (e == cudaSuccess) e = setup_one_fp8<true, 4>();
     if (e == cudaSuccess) e = setup_one_fp8<false, 8>();
     if (e == cudaSuccess) e = setup_one_fp8<true, 8>();
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(decode_fp8t_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * kWarpSmemT);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(decode_fp8t_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * kWarpSmemT);
     return e;
 }
 
@@ -488,8 +759,15 @@ cudaError_t launch_decode_fp8(const DecodeParams& p, int n_items, int warps, cud
     pp.gdc_wait = (overlap == 2) ? 0 : (overlap == 3) ? 2 : 1;
     const bool hi = p.G > 8;
     cudaError_t e;
-    if (warps == 8) e = hi ? cudaLaunchKernelEx(&cfg, decode_fp8_kernel<true, 8>, pp) : cudaLaunchKernelEx(&cfg, decode_fp8_kernel<false, 8>, pp);
-    else e = hi ? cudaLaunchKernelEx(&cfg, decode_fp8_kernel<true, 4>, pp) : cudaLaunchKernelEx(&cfg, decode_fp8_kernel<false, 4>, pp);
+    if (!hi) {
+        // groups of up to eight query heads: the transposed kernel
+        cfg.dynamicSmemBytes = warps * kWarpSmemT;
+        e = warps == 8 ? cudaLaunchKernelEx(&cfg, decode_fp8t_kernel<8>, pp) : cudaLaunchKernelEx(&cfg, decode_fp8t_kernel<4>, pp);
+    } else if (warps == 8) {
+        e = cudaLaunchKernelEx(&cfg, decode_fp8_kernel<true, 8>, pp);
+    } else {
+        e = cudaLaunchKernelEx(&cfg, decode_fp8_kernel<true, 4>, pp);
+    }
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
 }

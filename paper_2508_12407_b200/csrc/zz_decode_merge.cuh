@@ -74,6 +74,12 @@ struct ColsFp8 {
     __device__ __forceinline__ static int col(int i, int tig, int e) { return (i >> 1) * 16 + tig * 4 + e * 2 + (i & 1); }
 };
 
+template <int kWarps, int HD>
+__device__ __forceinline__ void finish_item_tail(const DecodeParams& p, unsigned char* smem, int* s_is_last_p, int item,
+                                                 int b, int hg, int nsplit, int len_old, bool advance_len,
+                                                 int* len_p, __nv_bfloat16* out_p, float* part_o_p, float* part_ml_p,
+                                                 unsigned int* counters_p, unsigned int* seq_counters_p);
+
 // Everything after a CTA's main loop.  `advance_len`: this launch makes the sequence one token longer
 // (the append fused into it, or the quantising append that ran just before it) and is the layer's last.
 template <int kWarps, int NR, class Cols, int HD = kD>
@@ -116,6 +122,23 @@ __device__ __forceinline__ void finish_item(const DecodeParams& p, unsigned char
         }
     }
     __syncthreads();
+    finish_item_tail<kWarps, HD>(p, smem, s_is_last_p, item, b, hg, nsplit, len_old, advance_len, len_p, out_p, part_o_p,
+                                 part_ml_p, counters_p, seq_counters_p);
+}
+
+// The part of the tail that starts from the warps' results staged in shared memory (sm_o [kWarps][16][HD]
+// fp32 rows of the group's query heads, then sm_ml [kWarps][16][2] = running maximum and sum), all warps
+// past a __syncthreads.
+template <int kWarps, int HD>
+__device__ __forceinline__ void finish_item_tail(const DecodeParams& p, unsigned char* smem, int* s_is_last_p, int item,
+                                                 int b, int hg, int nsplit, int len_old, bool advance_len,
+                                                 int* len_p, __nv_bfloat16* out_p, float* part_o_p, float* part_ml_p,
+                                                 unsigned int* counters_p, unsigned int* seq_counters_p) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = p.G;
+    int& s_is_last = *s_is_last_p;
+    float* sm_o = reinterpret_cast<float*>(smem);                  // [kWarps][16][HD]
+    float* sm_ml = sm_o + kWarps * 16 * HD;                        // [kWarps][16][2]
 
     const long long pair = (long long)b * p.Hg + hg;
     __nv_bfloat16* outb = out_p + ((long long)b * p.q_tok_stride) + (long long)(p.q_head0 + hg * G) * HD;
