@@ -221,3 +221,61 @@ def test_export_import_round_trip_and_refusals():
         binding.ZigzagCache(1, 1, 4, 2, 4, 8, [1], [40], 64, kv_fp8=True, pool_pages=4)
     assert e.value.status == binding.ZZ_ERR_UNSUPPORTED
     cache.close()
+
+
+def test_replayed_steps_on_fp8_stores_and_refusal_when_full():
+    """Decode steps of an FP8 cache replayed from a CUDA graph (quantising append + attention per step):
+    outputs against the oracle, stores bit for bit, and one replay beyond the reserved room is refused
+    on the device without touching a store."""
+    L, B, Hq, Hkv, S, W = 2, 2, 8, 2, 16, 48
+    kinds = [1, 0]
+    lens = [1500, 300]
+    n_replay = 20
+    scale = 1.0 / np.sqrt(D)
+    cap = [n + n_replay for n in lens]
+    cache = binding.ZigzagCache(L, B, Hq, Hkv, S, W, kinds, cap, 4096, kv_fp8=True)
+    w = inputs.Workload("f8g", L, B, Hq, Hkv, D, S, W, 1, 0, 0, n_replay, seed=808)
+    orc = [[Fp8Seq(Hkv, S, W, cap[b], [kinds[l]] * Hkv) for b in range(B)] for l in range(L)]
+    for l in range(L):
+        ks, vs = [], []
+        for b in range(B):
+            _, k, v = inputs.qkv_bf16(w, l, b, 0, lens[b])
+            orc[l][b].append(k, v)
+            ks.append(k); vs.append(v)
+        cache.kv_append(l, to_dev(np.concatenate(ks)), to_dev(np.concatenate(vs)), lens)
+    cache.reserve(n_replay)
+    sq = torch.zeros((L, B, Hq, D), dtype=torch.bfloat16, device="cuda:0")
+    sk = torch.zeros((L, B, Hkv, D), dtype=torch.bfloat16, device="cuda:0")
+    sv, so = torch.zeros_like(sk), torch.zeros_like(sq)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        cache.decode_step_all(sq, sk, sv, so)
+    for i in range(n_replay):
+        q = np.zeros((L, B, Hq, D), np.uint16); k = np.zeros((L, B, Hkv, D), np.uint16); v = np.zeros_like(k)
+        for l in range(L):
+            for b in range(B):
+                qq, kk, vv = inputs.qkv_bf16(w, l, b, lens[b] + i, 1)
+                q[l, b], k[l, b], v[l, b] = qq[0], kk[0], vv[0]
+                orc[l][b].append(kk, vv)
+        sq.copy_(to_dev(q)); sk.copy_(to_dev(k)); sv.copy_(to_dev(v))
+        g.replay()
+        got = to_bits(so)
+        if i % 6 == 0 or i == n_replay - 1:
+            for l in range(L):
+                for b in range(B):
+                    assert_close(got[l, b:b + 1], orc[l][b].decode_row(q[l, b:b + 1], scale), f"replay {i} layer {l} seq {b}")
+    torch.cuda.synchronize()
+    assert cache.last_status() == 0
+    cache.sync_len()
+    for l in range(L):
+        for b in range(B):
+            assert cache.len(l, b) == lens[b] + n_replay
+            check_stores(cache, l, b, orc[l][b])
+    before = [cache.export_fp8(0, b) for b in range(B)]
+    g.replay()                                   # the retrieval stores are full
+    torch.cuda.synchronize()
+    assert cache.last_status() == binding.ZZ_ERR_CAPACITY
+    after = [cache.export_fp8(0, b) for b in range(B)]
+    for x, y in zip(before, after):
+        assert x[4] == y[4] and all(np.array_equal(a, b_) for a, b_ in zip(x[:4], y[:4]))
+    cache.close()
