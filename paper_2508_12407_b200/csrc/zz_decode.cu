@@ -42,8 +42,7 @@ __device__ __forceinline__ void load_block(uint32_t stage_k, uint32_t stage_v, c
                                            const __nv_bfloat16* vbase, int tok0, int tok_end, int lane,
                                            int new_slot, const __nv_bfloat16* knew, const __nv_bfloat16* vnew,
                                            uint64_t policy) {
-    constexpr int kRowB = HD * 2;              // bytes of a row
-    constexpr int kPieces = HD / 8;            // 16-byte pieces of a row
+    constexpr int kRowB = HD * 2;              // bytes of a row (HD / 8 sixteen-byte pieces)
     if (HD == 64) {
         // 128-byte rows: lane -> (row it * 4 + lane / 8, piece lane % 8), pieces XOR-swizzled by row
         const bool whole = tok0 + kBlk <= tok_end && (new_slot < tok0 || new_slot >= tok0 + kBlk);

@@ -91,7 +91,6 @@ __device__ __forceinline__ void finish_item(const DecodeParams& p, unsigned char
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int grp = lane >> 2, tig = lane & 3;
     const int G = p.G;
-    int& s_is_last = *s_is_last_p;
     // ---- merge the warps of this CTA ---------------------------------------------------------
 #pragma unroll
     for (int hf = 0; hf < NR; ++hf) {

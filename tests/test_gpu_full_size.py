@@ -29,7 +29,7 @@ def _rows(P, c, S, W, n_extra, rng):
 
 
 def run_full(w: inputs.Workload, kinds, lens, chunk, n_decode, kvk=None, prefilled=False, rows_per_call=6,
-             decode_seqs=None, same_prompt_all_layers=False, paged=False):
+             decode_seqs=None, same_prompt_all_layers=False, paged=False, fp8=False):
     L, B, Hq, Hkv, S, W = len(kinds), len(lens), w.n_q_heads, w.n_kv_heads, w.sink, w.recent
     import torch
     scale = w.scale
@@ -39,13 +39,25 @@ def run_full(w: inputs.Workload, kinds, lens, chunk, n_decode, kvk=None, prefill
     kk = np.asarray(kvk).reshape(L, Hkv) if kvk is not None else np.repeat(np.asarray(kinds)[:, None], Hkv, axis=1)
     # paged: a pool with exactly the pages the run needs (one per retrieval head per 128 tokens)
     pool = int(kk.sum()) * sum((int(n) + n_decode + 127) // 128 for n in lens) if paged else 0
-    cache = binding.ZigzagCache(L, B, Hq, Hkv, S, W, kinds, cap, max_new, kvhead_is_retrieval=kvk, pool_pages=pool)
+    cache = binding.ZigzagCache(L, B, Hq, Hkv, S, W, kinds, cap, max_new, kvhead_is_retrieval=kvk, pool_pages=pool,
+                                kv_fp8=fp8)
     kv_kinds = [list(np.asarray(kvk).reshape(L, Hkv)[l]) if kvk is not None else [int(kinds[l])] * Hkv
                 for l in range(L)]
     hist_k = [[np.zeros((cap[b], Hkv, D), np.uint16) for b in range(B)] for l in range(L)]
     hist_v = [[np.zeros((cap[b], Hkv, D), np.uint16) for b in range(B)] for l in range(L)]
     pos = np.zeros((L, B), dtype=np.int64)
     shared = {}
+
+    def as_stored(l, x):
+        """Rows as they read back from the stores: FP8 retrieval heads hold quantised values (exactly bf16 numbers)."""
+        if not fp8:
+            return x
+        y = x.copy()
+        for h in range(Hkv):
+            if kv_kinds[l][h]:
+                y[:, h] = oracle.fp8_stored_as_bf16_bits(np.ascontiguousarray(x[:, h]))
+        return y
+
     for l in range(L):
         step = chunk if chunk else 8192
         done = np.zeros(B, dtype=np.int64)
@@ -66,6 +78,7 @@ def run_full(w: inputs.Workload, kinds, lens, chunk, n_decode, kvk=None, prefill
                     q, k, v = inputs.qkv_bf16(w, lk, b, int(done[b]), n_new[b])
                     if same_prompt_all_layers:
                         shared[(b, int(done[b]))] = (q, k, v)
+                # the chunk attends to itself as given; what it leaves in the history is what the stores hold
                 hist_k[l][b][done[b]:done[b] + n_new[b]] = k
                 hist_v[l][b][done[b]:done[b] + n_new[b]] = v
                 qs.append(q); ks.append(k); vs.append(v)
@@ -88,6 +101,13 @@ def run_full(w: inputs.Workload, kinds, lens, chunk, n_decode, kvk=None, prefill
                     off += c; i += 1
                 del dq, out
             cache.kv_append(l, dk, dv, n_new)
+            if fp8:
+                i = 0
+                for b in range(B):
+                    if n_new[b]:
+                        sl = slice(int(done[b]), int(done[b]) + n_new[b])
+                        hist_k[l][b][sl] = as_stored(l, ks[i]); hist_v[l][b][sl] = as_stored(l, vs[i])
+                        i += 1
             done += np.asarray(n_new)
         pos[l] = done
     # decode steps through the whole-stack call the benchmark times
@@ -98,7 +118,7 @@ def run_full(w: inputs.Workload, kinds, lens, chunk, n_decode, kvk=None, prefill
             for b in range(B):
                 qq, kk, vv = inputs.qkv_bf16(w, l, b, int(pos[l, b]), 1)
                 q[l, b], k[l, b], v[l, b] = qq[0], kk[0], vv[0]
-                hist_k[l][b][pos[l, b]] = kk[0]; hist_v[l][b][pos[l, b]] = vv[0]
+                hist_k[l][b][pos[l, b]] = as_stored(l, kk)[0]; hist_v[l][b][pos[l, b]] = as_stored(l, vv)[0]
         dq, dk, dv = to_dev(q), to_dev(k), to_dev(v)
         out = torch.zeros_like(dq)
         cache.decode_step_all(dq, dk, dv, out)
@@ -124,7 +144,16 @@ def run_full(w: inputs.Workload, kinds, lens, chunk, n_decode, kvk=None, prefill
                 gk, gv, gpos, glen = cache.export(l, b, binding.KIND_STREAMING)
                 assert glen == n and np.array_equal(gpos, ring.pos)
                 assert np.array_equal(gk, ring.k) and np.array_equal(gv, ring.v)
-            if r_heads:
+            if r_heads and fp8:
+                # the history holds the values the oracle's quantiser leaves in a store: the GPU's codes and scale
+                # bytes must decode to exactly those (the codes themselves are compared in tests/test_gpu_fp8.py)
+                gk, gv, gks, gvs, glen = cache.export_fp8(l, b)
+                assert glen == n
+                sl = slice(max(0, n - 3000), n)
+                for got_c, got_s, hist in ((gk, gks, hist_k), (gv, gvs, hist_v)):
+                    want_vals = inputs.bf16_bits_to_f64(np.ascontiguousarray(hist[l][b][sl][:, r_heads].transpose(1, 0, 2)))
+                    assert np.array_equal(oracle.fp8_dequantize_rows(got_c[:, sl], got_s[:, sl]), want_vals)
+            elif r_heads:
                 gk, gv, gpos, glen = cache.export(l, b, binding.KIND_RETRIEVAL)
                 assert glen == n and np.array_equal(gpos[:n], np.arange(n)) and (gpos[n:] == -1).all()
                 sl = slice(max(0, n - 3000), n)
@@ -169,3 +198,20 @@ def test_cfg4_ragged_batch16_paged_stores():
     w = inputs.WORKLOADS["cfg4"]
     lens = [int(x) for x in inputs.ragged_lengths(w)]
     run_full(w, [1, 0], lens, 0, 3, prefilled=True, decode_seqs=[0, 5, 11, 15], paged=True)
+
+
+def test_cfg2_32k_fp8_retrieval_stores():
+    w = inputs.WORKLOADS["cfg2"]
+    run_full(w, [1, 0, 1], [w.prefill_len], w.prefill_chunk, 4, fp8=True)
+
+
+def test_cfg4_ragged_batch16_fp8_retrieval_stores():
+    w = inputs.WORKLOADS["cfg4"]
+    lens = [int(x) for x in inputs.ragged_lengths(w)]
+    run_full(w, [1, 0], lens, 0, 3, prefilled=True, decode_seqs=[0, 5, 11, 15], fp8=True)
+
+
+def test_cfg3_chunked_prefill_over_fp8_stores():
+    # 8K chunks attending to an FP8 store that grows to 64K: the bf16 scratch path of the prefill
+    w = inputs.WORKLOADS["cfg3"]
+    run_full(w, [1, 0], [65536], w.prefill_chunk, 2, rows_per_call=1, fp8=True)
