@@ -139,6 +139,8 @@ struct zz_cache {
     int decode_overlap;
     int decode_multi_waves;
     bool last_nowait;   // the last launch did not wait for its predecessor: the next one must be an ordinary launch
+    int fresh_layer;    // layer whose store rows below the host length the last launch may still be writing
+                        // (-1: none, -2: any): no launch fetches them before it has waited for that launch
     bool has_mixed;
     // paged retrieval stores
     bool fp8;                         // retrieval stores hold E4M3 codes + a scale byte per token and head
@@ -428,6 +430,7 @@ int reserve_pages(zz_cache* c, int l0, int l1, const int32_t* add, cudaStream_t 
     if (!flush()) return ZZ_ERR_CUDA;
     c->table_dirty = true;
     c->last_nowait = false;   // the table writes were ordinary launches
+    c->fresh_layer = -2;
     return ZZ_OK;
 }
 
@@ -494,6 +497,17 @@ int launch_decode_group(zz_cache* c, int layer, int kind, const __nv_bfloat16* q
     if (c->table_dirty) overlap = 0;
     c->table_dirty = false;
     c->last_nowait = (overlap == 2);
+    // Rows a launch may fetch before it waits for its predecessor: those of a contiguous retrieval
+    // store that were complete before the predecessor began.  The host length counts them, unless the
+    // predecessor itself appended to this layer.
+    const bool early = overlap == 3 && kind == ZZ_KIND_RETRIEVAL && !fp8 && !c->paged && !d_layer_ids &&
+                       (c->fresh_layer == -1 || (c->fresh_layer >= 0 && c->fresh_layer != layer));
+    for (int b = 0; b < c->B; ++b) p.early_len[b] = early ? c->len[(size_t)layer * c->B + b] : 0;
+    // what this launch leaves behind for the next one: a launch that does not wait at entry may still
+    // run beside its own predecessor, so nothing is known to be complete after it
+    if (overlap == 1 || overlap == 2 || d_layer_ids) c->fresh_layer = -2;
+    else if (with_token) c->fresh_layer = layer;
+    else c->fresh_layer = -1;
     if (d_layer_ids) {
         // one launch for n_multi layers with identical lengths: `layer` stands for all of them in the
         // plan above; every per-layer pointer becomes the layer-0 pointer plus a stride per layer
@@ -550,6 +564,7 @@ int quant_append(zz_cache* c, int layer, const __nv_bfloat16* k, const __nv_bflo
     }
     zz::prof_begin(zz::kProfAppend, st);
     c->last_nowait = false;
+    c->fresh_layer = d_layer_ids ? -2 : layer;
     const cudaError_t e = zz::launch_quant_append(p, worst, d_layer_ids ? n_layers : 1, st);
     zz::prof_end(zz::kProfAppend, st);
     return e == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
@@ -577,6 +592,7 @@ int regroup(zz_cache* c, int layer, const __nv_bfloat16* src, __nv_bfloat16* dst
     zz::prof_begin(zz::kProfRegroup, st);
     const cudaError_t e = zz::launch_regroup(g, st, c->last_nowait ? 0 : 1);
     c->last_nowait = false;
+    c->fresh_layer = -2;     // (the regroup launch may itself run beside its predecessor)
     zz::prof_end(zz::kProfRegroup, st);
     return e == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
 }
@@ -646,6 +662,7 @@ int launch_prefill_group(zz_cache* c, int layer, int kind, const CUtensorMap* tq
     const int pk = (kind == ZZ_KIND_RETRIEVAL) ? zz::kProfPrefillR : zz::kProfPrefillS;
     zz::prof_begin(pk, st);
     c->last_nowait = false;   // an ordinary launch: full stream order
+    c->fresh_layer = -1;
     const cudaError_t e = zz::launch_prefill(p, tq, tk, tv, &c->tmap_arena, (int)items, st);
     zz::prof_end(pk, st);
     return e == cudaSuccess ? ZZ_OK : ZZ_ERR_CUDA;
@@ -734,6 +751,7 @@ static int create_impl(const zz_config_t* cfg, long long pool_pages, void* d_are
     c->decode_short_tokens = 384;
     c->decode_overlap = 3;
     c->last_nowait = false;
+    c->fresh_layer = -1;
     c->decode_multi_waves = 8;
     c->fp8 = cfg->retrieval_kv_fp8 != 0;
     compute_layout(cfg, &c->lay, &c->desc, pool_pages, &c->desc_scratch);
@@ -833,6 +851,7 @@ int zz_cache_reset(zz_cache_t* c, int seq, void* stream) {
     if (!c || seq < -1 || seq >= c->B) return ZZ_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     c->last_nowait = false;
+    c->fresh_layer = -1;
     if (zz::launch_reset(c->d_len(0), c->d_pos(0), c->L, c->B, c->ring, seq, st) != cudaSuccess)
         return ZZ_ERR_CUDA;
     zz::TableUpdate u;
@@ -969,6 +988,7 @@ int zz_kv_append(zz_cache_t* c, int layer, const void* d_k, const void* d_v, con
     if (gx > 0x7fffffffLL) return ZZ_ERR_UNSUPPORTED;
     zz::prof_begin(zz::kProfAppend, static_cast<cudaStream_t>(stream));
     c->last_nowait = false;
+    c->fresh_layer = layer;
     const cudaError_t ae = zz::launch_append(p, (int)gx, static_cast<cudaStream_t>(stream));
     zz::prof_end(zz::kProfAppend, static_cast<cudaStream_t>(stream));
     if (ae != cudaSuccess) return ZZ_ERR_CUDA;

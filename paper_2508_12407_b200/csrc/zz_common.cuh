@@ -107,6 +107,9 @@ struct DecodeParams {
                              // 2: wait at kernel entry; 0: never
     int split_start[ZZ_MAX_BATCH + 1];  // prefix sum of per-sequence split counts
     int chunk[ZZ_MAX_BATCH];            // tokens per split of each sequence
+    int early_len[ZZ_MAX_BATCH];        // rows of each sequence's retrieval store that were complete before the
+                                        // previous launch in the stream began (0: none known): a launch that
+                                        // waits at entry may fetch blocks below this length before it waits
     SeqDesc sd[ZZ_MAX_BATCH];           // store addresses of every sequence of this layer
     // several layers in one launch (blockIdx.y): layer_ids[y] is the layer, every per-layer pointer
     // above is then the layer-0 pointer and advances by these strides (elements) per layer; the

@@ -110,13 +110,8 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int grp = lane >> 2, tig = lane & 3;
 
-    // Programmatic dependent launch (no-ops in an ordinary launch): the next launch in the stream
-    // may start as soon as every CTA of this one is running, and fills the SMs this launch leaves
-    // idle in its tail.  A launch that shares anything with its predecessor (gdc_wait) touches it
-    // only after griddepcontrol.wait below; the layers of one decode step share nothing (own
-    // stores, lengths, split workspace and output slice) and run without that wait.
-    if (p.gdc_wait == 2) asm volatile("griddepcontrol.wait;" ::: "memory");   // before anything is read
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // (a launch that waits at entry lets its dependents go after that wait, further down)
+    if (p.gdc_wait != 2) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---- which layer (a launch may cover several layers of a decode step: blockIdx.y) -----------
     const int li = p.layer_ids ? p.layer_ids[blockIdx.y] : 0;
@@ -132,7 +127,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     float* const part_o_p = p.part_o + (long long)li * p.st_part * HD;
     float* const part_ml_p = p.part_ml + (long long)li * p.st_part * 2;
 
-    // ---- which work item -----------------------------------------------------------
+    // ---- which work item (launch parameters only) ----------------------------------------
     const int item = blockIdx.x;
     int b = 0;
     while (b + 1 < p.B && item >= p.split_start[b + 1] * p.Hg) ++b;
@@ -148,16 +143,71 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
         return;
     }
 
-    const bool fused = k_new_p != nullptr;
-    const int len_old = len_p[b];
+    // (read beside the store addresses unless the launch has to wait first)
+    const int len_nowait = (p.gdc_wait != 2) ? len_p[b] : 0;
+    // store addresses: written when the cache was created, never by a launch
     const SeqDesc sd = p.layer_ids ? p.desc_table[(long long)li * p.B + b] : p.sd[b];
-    const int len = len_old + (fused ? 1 : 0);
-    const int n = (p.kind == ZZ_KIND_RETRIEVAL) ? len : min(len, p.ring);
     const long long slots_per_head = (p.kind == ZZ_KIND_RETRIEVAL) ? sd.cap : p.ring;
     // paged retrieval store: the bases are the pool's; each 16-token block adds its page's offset
     constexpr bool paged = kPaged;
     __nv_bfloat16* kbase = p.arena + sd.k_off[p.kind] + (paged ? 0ll : (long long)hg * slots_per_head * HD);
     __nv_bfloat16* vbase = p.arena + sd.v_off[p.kind] + (paged ? 0ll : (long long)hg * slots_per_head * HD);
+    const uint32_t wbase = smem_u32(smem) + warp * kWarpSmem;
+    // L2 policy of the K/V loads: a retrieval store is streamed once per step and should not push
+    // anything out of the L2 (evict first); the rings of the streaming layers are read again by the
+    // next step and together fit the L2 (evict last)
+    uint64_t l2_policy;
+    if (p.kind == ZZ_KIND_RETRIEVAL)
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(l2_policy));
+    else
+        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(l2_policy));
+
+    // Programmatic dependent launch (no-ops in an ordinary launch): the next launch in the stream
+    // may start as soon as every CTA of this one is running, and fills the SMs this launch leaves
+    // idle in its tail.  A launch that shares anything with its predecessor (gdc_wait) touches it
+    // only after griddepcontrol.wait below; the layers of one decode step share nothing (own
+    // stores, lengths, split workspace and output slice) and run without that wait.
+    //
+    // A launch that waits at entry (gdc_wait == 2) still has something it may do first.  A retrieval
+    // store is append-only, so the rows that were complete before the previous launch began
+    // (early_len, from the host) cannot change under it: the first stages of the K/V pipeline are
+    // fetched before the wait, while the previous launch drains, whenever their blocks lie wholly
+    // below that length.  The plan (chunk, split_start) is in the launch parameters, so the blocks
+    // are known without the device length; the length, q and the step's token are read after the wait.
+    unsigned pre = 0;           // bit s: stage s of the prologue is already in flight
+    if (p.gdc_wait == 2) {
+        if constexpr (!kPaged) {
+            if (p.kind == ZZ_KIND_RETRIEVAL) {
+                const int ne = p.early_len[b];
+                const int e0 = split * p.chunk[b];
+                const int e1 = (split == nsplit - 1) ? ne : min(ne, e0 + p.chunk[b]);
+#pragma unroll
+                for (int s = 0; s < kStages - 1; ++s) {
+                    const int tok0 = e0 + (warp + s * kWarps) * kBlk;
+                    if (tok0 + kBlk <= e1) {
+                        load_block<HD>(wbase + s * 2 * kStageBytes, wbase + s * 2 * kStageBytes + kStageBytes, kbase,
+                                       vbase, tok0, e1, lane, -1, nullptr, nullptr, l2_policy);
+                        pre |= 1u << s;
+                    }
+                    cp_async_commit();
+                }
+            }
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // before anything a launch may have written is read
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
+
+    const bool fused = k_new_p != nullptr;
+    const int len_old = (p.gdc_wait != 2) ? len_nowait : len_p[b];
+    if (pre != 0 && len_old < p.early_len[b]) {
+        // the store is shorter than the host believed (lengths reset under a replayed launch): what was
+        // fetched early may lie past its end; let those copies land and fill the stages again below
+        cp_async_wait<0>();
+        __syncwarp();
+        pre = 0;
+    }
+    const int len = len_old + (fused ? 1 : 0);
+    const int n = (p.kind == ZZ_KIND_RETRIEVAL) ? len : min(len, p.ring);
     const int* const tbl = paged ? p.page_table + sd.tbl + hg : nullptr;   // entry of page g: tbl[g * Hg]
     int new_slot = -1;
     const __nv_bfloat16* knew = nullptr;
@@ -171,6 +221,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
         if (paged && room) room = tbl[(len_old >> 7) * p.Hg] >= 0;
         if (!room) {
             if (threadIdx.x == 0) atomicCAS(p.status, 0, ZZ_ERR_CAPACITY);
+            cp_async_wait<0>();     // stages fetched before the wait
             return;
         }
     }
@@ -225,16 +276,6 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     float m_run[2] = {-INFINITY, -INFINITY};
     float l_run[2] = {0.f, 0.f};
 
-    const uint32_t wbase = smem_u32(smem) + warp * kWarpSmem;
-    // L2 policy of the K/V loads: a retrieval store is streamed once per step and should not push
-    // anything out of the L2 (evict first); the rings of the streaming layers are read again by the
-    // next step and together fit the L2 (evict last)
-    uint64_t l2_policy;
-    if (p.kind == ZZ_KIND_RETRIEVAL)
-        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(l2_policy));
-    else
-        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(l2_policy));
-
     // Paged store: lane i holds the page of token block pg0 + i (32 pages = 4096 tokens); a block's
     // page is a shuffle away, the window is reloaded when the warp walks past it.  Blocks start at
     // multiples of 16 tokens (the split plan of a paged cache guarantees it), so a block never
@@ -256,7 +297,7 @@ __global__ void __launch_bounds__(kWarps * 32, 8 / kWarps) decode_kernel(const D
     // prologue: fill kStages-1 stages
 #pragma unroll
     for (int s = 0; s < kStages - 1; ++s) {
-        if (s < my_blocks) {
+        if (s < my_blocks && !((pre >> s) & 1u)) {
             const int tok0 = s0 + (warp + s * kWarps) * kBlk;
             const long long po = page_off(tok0);
             load_block<HD>(wbase + s * 2 * kStageBytes, wbase + s * 2 * kStageBytes + kStageBytes, kbase + po, vbase + po,

@@ -109,3 +109,72 @@ def test_reserve_refuses_beyond_capacity_or_pool():
     cache.reserve(57)                                            # 257 tokens: a third block
     assert cache.pages() == (6, 0)
     cache.close()
+
+
+def test_replayed_per_layer_steps_and_a_replay_after_reset():
+    """One zz_decode_step per layer (what a model calls between its own kernels), captured once:
+    consecutive retrieval layers let a launch fetch the first blocks of its store while the launch
+    before it drains.  The graph is replayed while the stores grow, then once more after the cache
+    was emptied: the captured launches then carry lengths the stores no longer have, and must fall
+    back to what the device says."""
+    import torch
+    L, B, Hq, Hkv, S, W = 4, 2, 8, 2, 16, 48
+    kinds = [1, 1, 0, 1]
+    lens = [3000, 700]
+    n_replay = 40
+    cap = [n + n_replay for n in lens]
+    cache = make(L, B, Hq, Hkv, S, W, kinds, cap, max_new=4096)
+    w = inputs.Workload("t", L, B, Hq, Hkv, D, S, W, 3, 0, 0, n_replay, seed=616)
+    new_orc = lambda: [[OracleSeq(Hkv, D, S, W, cap[b], [kinds[l]] * Hkv) for b in range(B)] for l in range(L)]
+    orc = new_orc()
+    _fill(cache, w, L, B, lens, orc)
+    cache.reserve(n_replay)
+    sq = torch.zeros((L, B, Hq, D), dtype=torch.bfloat16, device="cuda:0")
+    sk = torch.zeros((L, B, Hkv, D), dtype=torch.bfloat16, device="cuda:0")
+    sv = torch.zeros_like(sk)
+    so = torch.zeros_like(sq)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for l in range(L):
+            cache.decode_step(l, sq[l], sk[l], sv[l], so[l])
+    scale = 1 / np.sqrt(D)
+
+    def replay(base, i, check):
+        q = np.zeros((L, B, Hq, D), np.uint16); k = np.zeros((L, B, Hkv, D), np.uint16); v = np.zeros_like(k)
+        for l in range(L):
+            for b in range(B):
+                qq, kk, vv = inputs.qkv_bf16(w, l, b, base[b] + i, 1)
+                q[l, b], k[l, b], v[l, b] = qq[0], kk[0], vv[0]
+                orc[l][b].append(kk, vv)
+        sq.copy_(to_dev(q)); sk.copy_(to_dev(k)); sv.copy_(to_dev(v))
+        g.replay()
+        got = to_bits(so)
+        if check:
+            for l in range(L):
+                for b in range(B):
+                    want = orc[l][b].rows(q[l, b:b + 1], [orc[l][b].len - 1], scale=scale)
+                    assert_close(got[l, b:b + 1], want, f"replay {i} layer {l} seq {b}")
+
+    for i in range(n_replay):
+        replay(lens, i, i % 7 == 0 or i == n_replay - 1)
+    torch.cuda.synchronize()
+    assert cache.last_status() == 0
+    cache.sync_len()
+    for l in range(L):
+        for b in range(B):
+            assert cache.len(l, b) == lens[b] + n_replay
+            check_export(cache, l, b, orc[l][b])
+
+    # the cache is emptied; the captured launches still carry the old lengths and split plan
+    cache.reset()
+    orc = new_orc()
+    for i in range(20):
+        replay([0, 0], i, True)
+    torch.cuda.synchronize()
+    assert cache.last_status() == 0
+    cache.sync_len()
+    for l in range(L):
+        for b in range(B):
+            assert cache.len(l, b) == 20
+            check_export(cache, l, b, orc[l][b])
+    cache.close()
