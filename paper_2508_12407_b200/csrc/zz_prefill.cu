@@ -66,7 +66,7 @@ struct Shared {
     uint64_t kv_empty[kPairs];
     uint64_t s_full[2];
     uint64_t p_full[2];
-    uint64_t o_full;
+    uint64_t o_full[2];        // per query tile: its last P V has completed
     uint32_t tmem_base;
     uint32_t poll_limit;       // probes a wait may spend before it gives up (kMaxPolls in the product kernels)
     int abort_flag;
@@ -352,7 +352,7 @@ __device__ __forceinline__ int item_index(int k, int n_items) {
     const int idx = k * g + ((k & 1) ? g - 1 - (int)blockIdx.x : (int)blockIdx.x);
     return idx < n_items ? idx : -1;
 }
-__device__ __forceinline__ Item get_item(const PrefillParams& p, int idx) {
+__device__ __forceinline__ Item get_item(const PrefillParams& p, int kind, int idx) {
     Item it;
     const int pairs = (p.G + 1) >> 1;
     const int per_tile = p.Hg * pairs;
@@ -369,7 +369,7 @@ __device__ __forceinline__ Item get_item(const PrefillParams& p, int idx) {
     it.r0 = it.qt * kTile;
     it.C = p.n_new[b];
     it.P = p.len[b];
-    it.plan = make_plan(p.kind, it.P, it.C, it.qt, p.S, p.W, p.ring);
+    it.plan = make_plan(kind, it.P, it.C, it.qt, p.S, p.W, p.ring);
     it.n_tiles = it.plan.n_total;
     return it;
 }
@@ -389,7 +389,9 @@ __device__ __forceinline__ int item_key(const PrefillParams& p, int idx) {
 // tokens; on 32K chunks the two time the same.
 // HD = head_dim: 128, or 64 (Q, K and V tiles are then one 64-column sub-tile, Q K^T has four MMA steps
 // instead of eight, P V has N = 64, and O takes 64 columns of tensor memory).
-template <bool kPersistent, int HD>
+// kStreaming: the kind of layer (compiled apart: a retrieval launch carries none of the ring and window
+// arithmetic, and the short items of a streaming launch end each query tile on a barrier of its own).
+template <bool kPersistent, int HD, bool kStreaming>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q,
                const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
@@ -403,6 +405,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
     const uint32_t sm_kv = smem_base + 2 * kTileBytes;     // kStages K/V tiles
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int kind = kStreaming ? ZZ_KIND_STREAMING : ZZ_KIND_RETRIEVAL;
 
     const int n_items = p.n_items;
     const uint32_t sm_epi = smem_base + 2 * kTileBytes + kStages * kTileBytes;   // output staging
@@ -419,7 +422,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
         const int g = (int)gridDim.x, full = n_items / g, rem = n_items % g;
         const int pos = (full & 1) ? g - 1 - (int)blockIdx.x : (int)blockIdx.x;
         n_mine = full + (pos < rem ? 1 : 0);
-        use_order = p.kind == ZZ_KIND_RETRIEVAL && n_mine > 2 && n_mine <= kMaxOrder && p.B * p.Hg <= kMaxOrderKeys &&
+        use_order = kind == ZZ_KIND_RETRIEVAL && n_mine > 2 && n_mine <= kMaxOrder && p.B * p.Hg <= kMaxOrderKeys &&
                     p.B * p.Hg > 1;
     }
     unsigned char* const smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -480,7 +483,8 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
             mbar_init(&sh.s_full[i], 1);
             mbar_init(&sh.p_full[i], 128);
         }
-        mbar_init(&sh.o_full, 1);
+        mbar_init(&sh.o_full[0], 1);
+        mbar_init(&sh.o_full[1], 1);
         sh.poll_limit = kMaxPolls;
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -507,14 +511,14 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                 if (!kPersistent && k > 0) break;
                 const int idx = my_item(k);
                 if (idx < 0) break;
-                const Item it = get_item(p, idx);
+                const Item it = get_item(p, kind, idx);
                 const SeqDesc sd = p.desc[it.b];
-                const long long slots_per_head = (p.kind == ZZ_KIND_RETRIEVAL) ? sd.cap : p.ring;
+                const long long slots_per_head = (kind == ZZ_KIND_RETRIEVAL) ? sd.cap : p.ring;
                 // paged retrieval store: a store tile is one page (tiles and pages are both 128 tokens)
-                const bool paged = p.page_table != nullptr && p.kind == ZZ_KIND_RETRIEVAL;
+                const bool paged = p.page_table != nullptr && kind == ZZ_KIND_RETRIEVAL;
                 const int* const tbl = paged ? p.page_table + sd.tbl + it.hg : nullptr;
-                const int k_row0 = (int)(sd.k_off[p.kind] / HD + (paged ? 0ll : (long long)it.hg * slots_per_head));
-                const int v_row0 = (int)(sd.v_off[p.kind] / HD + (paged ? 0ll : (long long)it.hg * slots_per_head));
+                const int k_row0 = (int)(sd.k_off[kind] / HD + (paged ? 0ll : (long long)it.hg * slots_per_head));
+                const int v_row0 = (int)(sd.v_off[kind] / HD + (paged ? 0ll : (long long)it.hg * slots_per_head));
                 const int src_head = p.head_list[p.kv_head0 + it.hg];
                 const int tok0 = p.tok_off[it.b];
                 const int qh = p.q_head0 + it.hg * p.G + it.g0;
@@ -578,7 +582,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                 if (!kPersistent && k > 0) break;
                 const int idx = my_item(k);
                 if (idx < 0) break;
-                const Item it = get_item(p, idx);
+                const Item it = get_item(p, kind, idx);
                 const int n_tiles = __shfl_sync(0xffffffffu, it.n_tiles, 0);
                 const bool active1 = it.active1;
                 const int n_act = active1 ? 2 : 1;
@@ -629,6 +633,11 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                             // Commits cost tensor-pipe time beyond the first one after an MMA group, so
                             // there is one per tile (its S) plus one per iteration (the K/V pair is free)
                             mma_commit_if(more, &sh.s_full[t]);
+                            // the tile's last P V: its O is final (in a streaming launch each query tile has
+                            // its own barrier, so the epilogue of one does not wait for the other's last
+                            // softmax; in a retrieval launch, whose items are long, one commit per item after
+                            // the loop keeps this instruction stream as short as it can be)
+                            if constexpr (kStreaming) mma_commit_if(more ^ 1u, &sh.o_full[t]);
                             mma_commit_if(last_of_iter, &sh.kv_empty[slot]);
                             // after the item's last Q K^T the Q buffer may take the next item's tiles
                             if (kPersistent) mma_commit_if((j + 2 == n_tiles) & last_of_iter, &sh.q_empty);
@@ -636,8 +645,10 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                         __syncwarp();
                     }
                 }
-                if (leader) mma_commit(&sh.o_full);
-                __syncwarp();
+                if constexpr (!kStreaming) {
+                    if (leader) mma_commit(&sh.o_full[0]);
+                    __syncwarp();
+                }
                 u_glob += n_tiles + 1;
                 ph[0] += n_tiles;
                 if (active1) ph[1] += n_tiles;
@@ -653,11 +664,12 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
         const uint32_t t_o = t_s + 128;
         const float sc = p.scale_log2;
         uint32_t ph = 0;                                // S/P tiles of this query tile handled so far
+        uint32_t n_done = 0;                            // items this warpgroup has finished
         for (int k = 0;; ++k) {
             if (!kPersistent && k > 0) break;
             const int item_idx = my_item(k);
             if (item_idx < 0) break;
-            const Item it = get_item(p, item_idx);
+            const Item it = get_item(p, kind, item_idx);
             if (t == 1 && !it.active1) continue;
             const int n_tiles = it.n_tiles, r0 = it.r0, C = it.C, P = it.P, b = it.b, hg = it.hg, g0 = it.g0;
             const TilePlan plan = it.plan;
@@ -672,7 +684,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                 // tile_masked: some entry of this 128 x 128 tile may be invisible (uniform over the
                 // CTA); vis[w] bit i: column 32 w + i is visible to this thread's row
                 bool tile_masked = true;
-                if (p.kind == ZZ_KIND_RETRIEVAL) {
+                if (kind == ZZ_KIND_RETRIEVAL) {
                     tile_masked = is_chunk ? (start + 127 > r0) : (plan.n_occ - start < 128);
                 } else if (is_chunk) {
                     // a chunk tile of a streaming layer is fully visible to all 128 rows if it lies
@@ -689,7 +701,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
                 tmem_wait_ld();
                 if (tile_masked) {
                     uint32_t vis[4];
-                    if (p.kind == ZZ_KIND_RETRIEVAL) {
+                    if (kind == ZZ_KIND_RETRIEVAL) {
                         // store rows past the store's length; causal inside the chunk
                         const int lim = is_chunk ? (rr - start + 1) : (plan.n_occ - start);
 #pragma unroll
@@ -856,7 +868,9 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
 
             // ---- epilogue: O / l -> bf16 -> global ---------------------------------------------------
             ph += n_tiles;
-            mbar_wait(&sh.o_full, k & 1, &sh, p.status);
+            if constexpr (kStreaming) mbar_wait(&sh.o_full[t], n_done & 1, &sh, p.status);
+            else mbar_wait(&sh.o_full[0], k & 1, &sh, p.status);
+            ++n_done;
             tc_fence_after();
             const float inv = 1.f / l_run;
             // The warp stages 16 of its 32 rows at a time in its 4 KB of shared memory (16-byte pieces
@@ -870,39 +884,79 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmap_q
             const int piece_r = lane % kPieces, half_r = lane / kPieces;
             const long long row0 = (long long)p.tok_off[b] + r0 + quarter * 32;
             __nv_bfloat16* obase = p.out + (long long)(p.q_head0 + hg * p.G + g0 + t) * HD + piece_r * 8;
-#pragma unroll 1
-            for (int h = 0; h < 2; ++h) {
-#pragma unroll 1
-                for (int c = 0; c < HD / 32; ++c) {
-                    float o[32];
-                    tmem_ld32(t_o + c * 32, o);
-                    tmem_wait_ld();
-                    if ((lane >> 4) == h) {
+            if constexpr (kStreaming) {
+              // the thread's whole row leaves tensor memory once, scaled and rounded into kPieces 16-byte pieces
+              uint32_t w[HD / 2];
+              {
+                  float o[HD];
+                  if constexpr (HD == 128) {
+                      tmem_ld128(t_o, o);
+                  } else {
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const uint32_t w0 = pack_bf16(o[8 * i + 0] * inv, o[8 * i + 1] * inv);
-                            const uint32_t w1 = pack_bf16(o[8 * i + 2] * inv, o[8 * i + 3] * inv);
-                            const uint32_t w2 = pack_bf16(o[8 * i + 4] * inv, o[8 * i + 5] * inv);
-                            const uint32_t w3 = pack_bf16(o[8 * i + 6] * inv, o[8 * i + 7] * inv);
-                            const uint32_t piece = (uint32_t)(c * 4 + i);
-                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                                         ::"r"(stage + (lane & 15) * kRowB + ((piece ^ (lane & (kPieces - 1))) << 4)),
-                                           "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
-                        }
-                    }
-                }
-                __syncwarp();
+                      for (int c = 0; c < HD / 32; ++c) tmem_ld32(t_o + c * 32, o + c * 32);
+                  }
+                  tmem_wait_ld();
+#pragma unroll
+                  for (int i = 0; i < HD / 2; ++i) w[i] = pack_bf16(o[2 * i] * inv, o[2 * i + 1] * inv);
+              }
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                  if ((lane >> 4) == h) {
+#pragma unroll
+                      for (int piece = 0; piece < kPieces; ++piece)
+                          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                                       ::"r"(stage + (lane & 15) * kRowB + ((piece ^ (lane & (kPieces - 1))) << 4)),
+                                         "r"(w[4 * piece]), "r"(w[4 * piece + 1]), "r"(w[4 * piece + 2]), "r"(w[4 * piece + 3])
+                                       : "memory");
+                  }
+                  __syncwarp();
 #pragma unroll 4
-                for (int i = 0; i < kPieces / 2; ++i) {
-                    const int sr = (32 / kPieces) * i + half_r;            // row inside the staged 16
-                    const int lr = 16 * h + sr;                            // row inside the warp's 32
-                    uint32_t w0, w1, w2, w3;
-                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
-                                 : "r"(stage + sr * kRowB + ((piece_r ^ (sr & (kPieces - 1))) << 4)) : "memory");
-                    if (r0 + quarter * 32 + lr < C)
-                        *reinterpret_cast<uint4*>(obase + (row0 + lr) * p.tok_stride) = make_uint4(w0, w1, w2, w3);
-                }
-                __syncwarp();
+                  for (int i = 0; i < kPieces / 2; ++i) {
+                      const int sr = (32 / kPieces) * i + half_r;            // row inside the staged 16
+                      const int lr = 16 * h + sr;                            // row inside the warp's 32
+                      uint32_t w0, w1, w2, w3;
+                      asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
+                                   : "r"(stage + sr * kRowB + ((piece_r ^ (sr & (kPieces - 1))) << 4)) : "memory");
+                      if (r0 + quarter * 32 + lr < C)
+                          *reinterpret_cast<uint4*>(obase + (row0 + lr) * p.tok_stride) = make_uint4(w0, w1, w2, w3);
+                  }
+                  __syncwarp();
+              }
+            } else {
+#pragma unroll 1
+              for (int h = 0; h < 2; ++h) {
+#pragma unroll 1
+                  for (int c = 0; c < HD / 32; ++c) {
+                      float o[32];
+                      tmem_ld32(t_o + c * 32, o);
+                      tmem_wait_ld();
+                      if ((lane >> 4) == h) {
+#pragma unroll
+                          for (int i = 0; i < 4; ++i) {
+                              const uint32_t w0 = pack_bf16(o[8 * i + 0] * inv, o[8 * i + 1] * inv);
+                              const uint32_t w1 = pack_bf16(o[8 * i + 2] * inv, o[8 * i + 3] * inv);
+                              const uint32_t w2 = pack_bf16(o[8 * i + 4] * inv, o[8 * i + 5] * inv);
+                              const uint32_t w3 = pack_bf16(o[8 * i + 6] * inv, o[8 * i + 7] * inv);
+                              const uint32_t piece = (uint32_t)(c * 4 + i);
+                              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                                           ::"r"(stage + (lane & 15) * kRowB + ((piece ^ (lane & (kPieces - 1))) << 4)),
+                                             "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+                          }
+                      }
+                  }
+                  __syncwarp();
+#pragma unroll 4
+                  for (int i = 0; i < kPieces / 2; ++i) {
+                      const int sr = (32 / kPieces) * i + half_r;            // row inside the staged 16
+                      const int lr = 16 * h + sr;                            // row inside the warp's 32
+                      uint32_t w0, w1, w2, w3;
+                      asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
+                                   : "r"(stage + sr * kRowB + ((piece_r ^ (sr & (kPieces - 1))) << 4)) : "memory");
+                      if (r0 + quarter * 32 + lr < C)
+                          *reinterpret_cast<uint4*>(obase + (row0 + lr) * p.tok_stride) = make_uint4(w0, w1, w2, w3);
+                  }
+                  __syncwarp();
+              }
             }
         }
     }
@@ -944,25 +998,33 @@ cudaError_t launch_wait_probe(int* status, unsigned int polls, int* gave_up, cud
 
 static int g_num_sms = 0;
 
+template <bool kPersistent, int HD>
+static cudaError_t set_smem() {
+    cudaError_t e = cudaFuncSetAttribute(prefill_kernel<kPersistent, HD, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(prefill_kernel<kPersistent, HD, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    return e;
+}
+
 cudaError_t prefill_setup() {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(prefill_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(prefill_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(prefill_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(prefill_kernel<false, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = set_smem<true, 128>();
+    if (e == cudaSuccess) e = set_smem<false, 128>();
+    if (e == cudaSuccess) e = set_smem<true, 64>();
+    if (e == cudaSuccess) e = set_smem<false, 64>();
     return e;
 }
 
 template <bool kPersistent, int HD>
 static void launch_one(int grid, const PrefillParams& pp, const void* tq, const void* tk, const void* tv, const void* ta,
                        cudaStream_t s) {
-    prefill_kernel<kPersistent, HD><<<grid, kThreads, kSmemBytes, s>>>(pp, *static_cast<const CUtensorMap*>(tq),
-                                                                     *static_cast<const CUtensorMap*>(tk),
-                                                                     *static_cast<const CUtensorMap*>(tv),
-                                                                     *static_cast<const CUtensorMap*>(ta));
+    const CUtensorMap &mq = *static_cast<const CUtensorMap*>(tq), &mk = *static_cast<const CUtensorMap*>(tk),
+                      &mv = *static_cast<const CUtensorMap*>(tv), &ma = *static_cast<const CUtensorMap*>(ta);
+    if (pp.kind == ZZ_KIND_STREAMING) prefill_kernel<kPersistent, HD, true><<<grid, kThreads, kSmemBytes, s>>>(pp, mq, mk, mv, ma);
+    else prefill_kernel<kPersistent, HD, false><<<grid, kThreads, kSmemBytes, s>>>(pp, mq, mk, mv, ma);
 }
 
 cudaError_t launch_prefill(const PrefillParams& p, const void* tq, const void* tk, const void* tv,
