@@ -262,9 +262,13 @@ class Arm:
                 self.cache.prefill_attn(l, self.pq[i], self.pk[i], self.pv[i], self.pout, self.n_new)
                 self.cache.kv_append(l, self.pk[i], self.pv[i], self.n_new)
 
-    def step(self, profile_period=0):
-        """One step; returns [event before prefill, after prefill, after decode, decode launches, replayed launches]."""
+    def step(self, profile_period=0, graph=None):
+        """One step; returns [event before prefill, after prefill, after decode, decode launches, replayed launches].
+        graph: decode steps replayed from a CUDA graph re-captured every `graph` steps (None: as --graph says)."""
         binding, torch, args = self.binding, self.torch, self.args
+        graph = args.graph if graph is None else graph
+        if graph and self.side is None:
+            self.side = torch.cuda.Stream(device=self.dev)
         marks = [self.ev(), self.ev(), self.ev()]
         if self.C:
             self.cache.reset()
@@ -281,14 +285,14 @@ class Arm:
         binding.profile_enable(profile_period * 64)
         lc = binding.launch_count()
         extra = 0
-        if args.graph:
-            # the decode step captured into a CUDA graph and replayed; re-captured every args.graph
+        if graph:
+            # the decode step captured into a CUDA graph and replayed; re-captured every `graph`
             # steps so that the frozen split plan stays close to the growing stores.  Capture,
             # instantiation and the length read-back are inside the timed region.
             binding.profile_enable(0)          # no tracer events inside a capture
             done = 0
             while done < self.steps_dec:
-                n = min(args.graph, self.steps_dec - done)
+                n = min(graph, self.steps_dec - done)
                 self.cache.reserve(n)
                 g = torch.cuda.CUDAGraph()
                 lc0 = binding.launch_count()
@@ -574,11 +578,14 @@ def e2e_decode(arm, n_steps=32):
                     f"out back), after the same prefill; a step here is one token per sequence through all layers"}
 
 
-def compare_arms(excl, mixed, n_pairs):
+def compare_arms(excl, mixed, n_pairs, n_pairs_graph=2):
     """Exclusive-layer stack against the mixed-head stack on the same tensors, in alternating steps
-    (so that clock and temperature drift hit both alike); per-step phase times and their spread."""
+    (so that clock and temperature drift hit both alike); per-step phase times and their spread.
+    Then the same with every decode step replayed from a CUDA graph of one step (captured once per
+    benchmark step, capture and instantiation inside the timed decode phase)."""
     import torch
     rows = {"exclusive": {"prefill_ms": [], "decode_ms": []}, "mixed": {"prefill_ms": [], "decode_ms": []}}
+    rows_g = {"exclusive": [], "mixed": []}
     launches = {}
     mixed.step(0)                     # one warm-up step of the arm that has not run yet
     for _ in range(n_pairs):
@@ -588,6 +595,11 @@ def compare_arms(excl, mixed, n_pairs):
             rows[name]["prefill_ms"].append(m[0].elapsed_time(m[1]))
             rows[name]["decode_ms"].append(m[1].elapsed_time(m[2]))
             launches[name] = m[3]
+    for _ in range(n_pairs_graph if excl.steps_dec else 0):
+        for name, arm in (("exclusive", excl), ("mixed", mixed)):
+            m = arm.step(0, graph=arm.steps_dec)
+            torch.cuda.synchronize()
+            rows_g[name].append(m[1].elapsed_time(m[2]))
     B, sd = excl.w.batch, excl.steps_dec
 
     def stats(xs):
@@ -606,6 +618,14 @@ def compare_arms(excl, mixed, n_pairs):
                 "median": float(np.median(per_pair)), "min": float(per_pair.min()), "max": float(per_pair.max()),
                 "exclusive_faster_in_pairs": int((per_pair > 0).sum()),
                 "step_to_step_spread_exclusive": float((e.max() - e.min()) / np.median(e))}
+    if rows_g["exclusive"]:
+        e, m = np.asarray(rows_g["exclusive"]), np.asarray(rows_g["mixed"])
+        out["decode_from_graph"] = {
+            "pairs": int(e.size),
+            "exclusive_us_per_token": stats([x * 1e3 / (B * sd) for x in e]),
+            "mixed_us_per_token": stats([x * 1e3 / (B * sd) for x in m]),
+            "margin_decode": {"median": float(np.median((m - e) / m)), "min": float(((m - e) / m).min()),
+                              "max": float(((m - e) / m).max()), "exclusive_faster_in_pairs": int((m > e).sum())}}
     return out
 
 
