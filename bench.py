@@ -173,7 +173,8 @@ def run_reference(args, w):
     line = {"metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
-            "config": {"workload": w.name, "note": "fp64 CPU oracle on a bounded sample of the workload"},
+            "config": dict(workload_config(w, args, int(os.environ.get("WORLD_SIZE", "1")), mixed=args.mixed),
+                           note="fp64 CPU oracle on a bounded sample of this workload (rank 0 only)"),
             "cpu_baseline": dict(cb, value=v),
             "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -489,20 +490,30 @@ def summary(arm, r, K, world, p, traffic):
     return out, roofs, dom
 
 
-def config_of(arm, world):
-    w = arm.w
-    a = arm.args
-    return {"workload": w.name + ("+mixed" if arm.mixed else "") + ("+paged" if a.paged else "") + ("+fp8kv" if a.kv == "fp8" else "") + (f"+graph{a.graph}" if a.graph else ""),
+def workload_config(w, a, world, mixed=False):
+    """What was run, from the workload's definition and the flags alone (both arms of the benchmark
+    describe their run with it)."""
+    kinds = inputs.layer_kinds(w)
+    kvk = inputs.mixed_kvhead_kinds(w, w.mixed_retrieval_kv_heads or w.n_kv_heads // 2) if mixed else None
+    lens = inputs.ragged_lengths(w)
+    C = w.prefill_chunk if w.prefill_len else 0
+    steps_dec = w.decode_steps if a.decode_steps < 0 else a.decode_steps
+    base = float(lens.sum()) if not C else float(w.batch) * w.prefill_len
+    return {"workload": w.name + ("+mixed" if mixed else "") + ("+paged" if a.paged else "") + ("+fp8kv" if a.kv == "fp8" else "") + (f"+graph{a.graph}" if a.graph else ""),
             "retrieval_kv": "fp8 e4m3 codes + one power-of-two scale byte per token and head" if a.kv == "fp8" else "bf16",
             "layers": w.n_layers, "batch": w.batch, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
-            "sink": w.sink, "recent": w.recent, "retrieval_layers": int(arm.kinds.sum()) if arm.kvk is None else None,
-            "retrieval_kv_heads_per_layer": None if arm.kvk is None else int(arm.kvk.sum() // w.n_layers),
-            "prefill_len": w.prefill_len, "prefill_chunk": arm.C, "decode_steps": arm.steps_dec,
+            "sink": w.sink, "recent": w.recent, "retrieval_layers": int(kinds.sum()) if kvk is None else None,
+            "retrieval_kv_heads_per_layer": None if kvk is None else int(kvk.sum() // w.n_layers),
+            "prefill_len": w.prefill_len, "prefill_chunk": C, "decode_steps": steps_dec,
             "decode_overlap": a.decode_overlap if a.decode_overlap >= 0 else 3,
-            "context": [int(x) for x in arm.lens] if not arm.C else w.prefill_len,
+            "context": [int(x) for x in lens] if not C else w.prefill_len,
             "l2": "per-layer inputs larger than L2 (KV per retrieval layer %.0f MB)" % (
-                2 * w.n_kv_heads * float(arm.work()["base_len"].sum()) * w.head_dim * 2 / 1e6),
+                2 * w.n_kv_heads * base * w.head_dim * 2 / 1e6),
             "parallelism": f"replicas x{world}" if world > 1 else "single GPU"}
+
+
+def config_of(arm, world):
+    return workload_config(arm.w, arm.args, world, mixed=arm.mixed)
 
 
 def per_layer_decode(arm, p, n_steps=32):
