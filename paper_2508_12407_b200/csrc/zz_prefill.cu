@@ -1,8 +1,8 @@
 // Prefill attention on the 5th-generation tensor cores: tcgen05.mma with the S = Q K^T and
 // O = P V accumulators in tensor memory, operands staged in shared memory by TMA.
 //
-// One kernel serves both kinds of layer.  A retrieval head visits every KV tile up to the
-// diagonal (causal flash attention); a streaming head visits only the tiles that can hold
+// One kernel template serves both kinds of layer (compiled once per kind).  A retrieval head visits
+// every KV tile up to the diagonal (causal flash attention); a streaming head visits only the tiles that can hold
 // visible keys -- the sink tiles and the local band -- and applies the token-exact
 // visibility rule inside them (block sparsity is an execution strategy, not the mask).
 // Keys come from two places: the store as it stood before the call (append-only rows, contiguous
